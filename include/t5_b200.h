@@ -1,0 +1,181 @@
+/*
+ * t5_b200.h -- C ABI of the B200 (sm_100a) library that runs one training step
+ * (forward and backward) of a T5.1.1-style Transformer, plus the two inference
+ * calls a model must expose.
+ *
+ * Where the operations come from: the paper's "Example Models" section names
+ * the models (T5 / T5.1.1 encoder-decoder, and a decoder-only configuration);
+ * its "Model Implementation" section says a model is wrapped so that it exposes
+ * a loss, an evaluation and an inference method; its "Task-based API" section
+ * says feature converters hand the model raw integer arrays (encoder-decoder
+ * or decoder-only layouts).  The paper prints no formula; the arithmetic is the
+ * public T5.1.1 definition, restated beside each call below.
+ *
+ * Conventions for every call
+ *  - Returns 0 on success or a negative T5_ERR_* code.  Nothing aborts, throws
+ *    or traps.  t5_last_error() returns a message for the last failure on the
+ *    handle (or for a failed t5_create when passed NULL).
+ *  - Pointers named d_* are DEVICE pointers owned by the caller; they must be
+ *    16-byte aligned.  Everything else is a host pointer.
+ *  - The library allocates no device memory.  All work is enqueued on the
+ *    caller's stream (a cudaStream_t passed as void*); no call synchronises
+ *    the device.
+ *  - Token id 0 is padding.  Segment ids are optional (NULL = one example per
+ *    row); segment id 0 marks padding in packed rows.  A position's "code" is
+ *    0 when its token is padding, else its segment id (1 if unpacked).  Query
+ *    i attends key j iff code_k[j] != 0 and code_q[i] == code_k[j] (and
+ *    j <= i in the decoder's self-attention).  A query with no valid key
+ *    produces a zero attention output.  Decoder codes come from the targets.
+ */
+#ifndef T5_B200_H_
+#define T5_B200_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define T5_ABI_VERSION 1
+
+#if defined(__GNUC__)
+#define T5_API __attribute__((visibility("default")))
+#else
+#define T5_API
+#endif
+
+enum {
+  T5_OK = 0,
+  T5_ERR_NULL = -1,         /* a required pointer is NULL */
+  T5_ERR_CONFIG = -2,       /* unsupported or inconsistent configuration */
+  T5_ERR_SHAPE = -3,        /* batch sizes outside the configured maxima */
+  T5_ERR_ALIGN = -4,        /* device pointer not 16-byte aligned */
+  T5_ERR_WORKSPACE = -5,    /* workspace smaller than t5_workspace_bytes() */
+  T5_ERR_CUDA = -6,         /* a CUDA runtime/driver call failed (see message) */
+  T5_ERR_DEVICE_TIMEOUT = -7, /* a bounded device-side wait ran out */
+  T5_ERR_ARG = -8           /* bad scalar argument */
+};
+
+/* Model and execution configuration (plain data). */
+typedef struct {
+  int32_t abi_version;      /* T5_ABI_VERSION */
+  int32_t arch;             /* 0 encoder-decoder, 1 decoder-only */
+  int32_t n_enc_layers, n_dec_layers;
+  int32_t d_model, n_heads, d_kv, d_ff, vocab;
+  int32_t rel_buckets, rel_max_distance;        /* 32, 128 */
+  int32_t max_batch, max_enc_len, max_dec_len;  /* workspace sizing */
+  float z_loss, rms_eps, attn_scale, logit_scale; /* 1e-4, 1e-6, 1.0, d_model^-1/2 */
+  int32_t dtype;            /* 0: float32 everywhere (validation mode);
+                               1: bfloat16 parameters/operands, float32 accumulation */
+  int32_t recompute;        /* activation policy: 0 keep everything, 1 recompute cheap
+                               element-wise pieces in the backward pass */
+  int32_t flags;            /* bit 0: use the plain SIMT GEMM/attention kernels also in
+                               bfloat16 mode (debugging aid) */
+} t5_config;
+
+/* One batch.  All pointers are device pointers to int32 arrays. */
+typedef struct {
+  int32_t B, Te, Td;
+  const int32_t* d_enc_tokens;       /* [B,Te]; NULL for decoder-only */
+  const int32_t* d_enc_segment_ids;  /* [B,Te] or NULL */
+  const int32_t* d_dec_targets;      /* [B,Td]; decoder inputs = targets shifted right
+                                        (0 at a row or segment start) */
+  const int32_t* d_dec_segment_ids;  /* [B,Td] or NULL */
+} t5_batch;
+
+typedef struct t5_handle t5_handle;
+
+/* Host-only: validates the configuration and builds the parameter manifest. */
+T5_API int t5_create(const t5_config* cfg, t5_handle** out);
+T5_API int t5_destroy(t5_handle* h);
+T5_API const char* t5_last_error(const t5_handle* h);
+
+/* Parameters live in ONE flat device buffer of t5_param_count() elements of
+ * the configured dtype (gradients: the same layout in float32).  Tensor i of
+ * t5_param_tensors() has `name`, element `offset`, and `shape`.  Names follow
+ * the paper's logical-axis idea ("Model Implementation" section):
+ *   token_embed [vocab, embed]; {enc,dec}.relbias [buckets, heads];
+ *   *.norm / *.final_norm [embed];
+ *   enc.L<i>.attn.{q,k,v} [heads*kv, embed]; .o [embed, heads*kv];
+ *   *.ffn.{wi0,wi1} [mlp, embed]; .wo [embed, mlp];
+ *   dec.L<i>.{self,cross}.* likewise.
+ * Dense weights are stored [out_features, in_features], row-major: a
+ * projection computes y[t, o] = sum_i x[t, i] * W[o, i]. */
+T5_API int t5_param_count(const t5_handle* h, int64_t* n_elements);
+T5_API int t5_param_tensors(const t5_handle* h, int32_t* n_tensors);
+T5_API int t5_param_manifest(const t5_handle* h, int32_t idx, char name[64], int64_t* offset,
+                      int32_t shape[4], int32_t* ndim);
+
+/* Bytes of scratch the step needs at the configured maxima. */
+T5_API int t5_workspace_bytes(const t5_handle* h, int64_t* bytes);
+
+/* Fills d_params: matrices, embedding and bias tables ~ N(0, stddev), norm
+ * scales = 1.  Counter-based: element e of the flat buffer is a function of
+ * (seed, e) only (splitmix64 hash -> two uniforms -> Box-Muller). */
+T5_API int t5_init_params(t5_handle* h, void* d_params, uint64_t seed, float stddev, void* stream);
+
+/* The loss method and its gradient ("Model Implementation" section: a model
+ * defines its loss).  With w_t = [target_t != 0], W = sum w:
+ *   x = E[tokens];  per layer: x += Attn(RMS(x)), x += FFN(RMS(x));
+ *   RMS(x) = x * (mean(x^2)+eps)^-1/2 * g;
+ *   Attn: softmax_j(attn_scale * q_i.k_j + table[bucket(j-i), head] + mask) v, then Wo;
+ *         encoder: bidirectional buckets; decoder self: causal, one-sided buckets;
+ *         cross-attention: keys/values from the encoder output, no bias;
+ *   FFN(y) = (gelu_tanh(y Wi0) * (y Wi1)) Wo;
+ *   logits = logit_scale * RMS(x_dec) E^T;  lse_t = log sum_v exp(logits_tv);
+ *   L = (1/W) sum_t w_t (lse_t - logits_t[target_t] + z_loss * lse_t^2).
+ * Writes d_loss4 = [L, cross-entropy part, z-loss part, W] (float32) and
+ * OVERWRITES d_grads (float32, parameter layout) with dL/dparams.
+ * W = 0 gives zero loss and zero gradients. */
+T5_API int t5_train_step_fwd_bwd(t5_handle* h, const void* d_params, const t5_batch* batch,
+                          float* d_grads, float* d_loss4, void* d_workspace,
+                          int64_t workspace_bytes, void* stream);
+
+/* Inference method, encoder half: d_enc_out [B,Te,d_model] in the configured
+ * dtype = the encoder stack's output after its final norm. */
+T5_API int t5_encode(t5_handle* h, const void* d_params, const t5_batch* batch, void* d_enc_out,
+              void* d_workspace, int64_t workspace_bytes, void* stream);
+
+/* Inference method, decoder half: teacher-forced logits [B,Td,vocab]
+ * (configured dtype) for the whole target sequence given d_enc_out (ignored
+ * for decoder-only).  batch->d_enc_tokens / segment ids supply the key mask of
+ * the cross-attention. */
+T5_API int t5_decode_logits(t5_handle* h, const void* d_params, const t5_batch* batch,
+                     const void* d_enc_out, void* d_logits, void* d_workspace,
+                     int64_t workspace_bytes, void* stream);
+
+/* Reads back the status word the kernels of the last call on this workspace
+ * left behind (their waits on TMA/tensor-core barriers are bounded; one that
+ * runs out records a code instead of spinning).  SYNCHRONISES the stream.
+ * Returns T5_OK or T5_ERR_DEVICE_TIMEOUT. */
+T5_API int t5_device_status(t5_handle* h, const void* d_workspace, void* stream);
+
+/* ---- single operations of the path, exported for element-wise parity tests ---- */
+
+/* Relative-position bucket (closed form, exact integer thresholds):
+ * d_out[i] = bucket(rel_lo + i) for i in [0, n), rel = key - query. */
+T5_API int t5_relpos_buckets(int32_t bidirectional, int32_t num_buckets, int32_t max_distance,
+                      int32_t rel_lo, int32_t n, int32_t* d_out, void* stream);
+
+/* Softmax cross-entropy with z-loss over rows of logits [n_rows, vocab]
+ * (dtype 0 float32 / 1 bfloat16), IN PLACE: on return d_logits holds
+ * dL/dlogits = (w/W)(p (1 + 2 z lse) - onehot).  d_W: device float holding W.
+ * d_sums[2] (float64, zeroed by the caller) accumulate sum w*ce and sum w*z*lse^2;
+ * d_lse [n_rows] receives lse. */
+T5_API int t5_xent_zloss(int32_t dtype, void* d_logits, const int32_t* d_targets, int32_t n_rows,
+                  int32_t vocab, float z_loss, const float* d_W, double* d_sums, float* d_lse,
+                  void* stream);
+
+/* D[M,N] = alpha * A * B (+ D when accumulate), bf16/f32 operands, f32 accumulation.
+ * a_kmajor: A is stored [M,K] (else [K,M]); b_kmajor: B is stored [N,K] (else [K,N]);
+ * lda/ldb/ldd are row strides in elements.  out_f32: D is float32, else the operand
+ * dtype.  impl 0 = SIMT kernel, 1 = tcgen05/TMEM/TMA kernel (bfloat16 only). */
+T5_API int t5_gemm(int32_t dtype, int32_t impl, int32_t M, int32_t N, int32_t K, float alpha,
+            const void* d_A, int32_t lda, int32_t a_kmajor, const void* d_B, int32_t ldb,
+            int32_t b_kmajor, void* d_D, int32_t ldd, int32_t out_f32, int32_t accumulate,
+            void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* T5_B200_H_ */

@@ -1,0 +1,220 @@
+"""ctypes binding of libt5b200.so: argument marshalling only.
+
+Every function here has the name of the C entry point it wraps (see
+include/t5_b200.h) and does no arithmetic of its own.  torch is used for
+device buffers and the current stream.  Loading fails loudly when the library
+has not been built; there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libt5b200.so")
+
+T5_ABI_VERSION = 1
+ERR_NAMES = {0: "T5_OK", -1: "T5_ERR_NULL", -2: "T5_ERR_CONFIG", -3: "T5_ERR_SHAPE", -4: "T5_ERR_ALIGN",
+             -5: "T5_ERR_WORKSPACE", -6: "T5_ERR_CUDA", -7: "T5_ERR_DEVICE_TIMEOUT", -8: "T5_ERR_ARG"}
+
+
+class t5_config(C.Structure):
+    _fields_ = [("abi_version", C.c_int32), ("arch", C.c_int32),
+                ("n_enc_layers", C.c_int32), ("n_dec_layers", C.c_int32),
+                ("d_model", C.c_int32), ("n_heads", C.c_int32), ("d_kv", C.c_int32),
+                ("d_ff", C.c_int32), ("vocab", C.c_int32),
+                ("rel_buckets", C.c_int32), ("rel_max_distance", C.c_int32),
+                ("max_batch", C.c_int32), ("max_enc_len", C.c_int32), ("max_dec_len", C.c_int32),
+                ("z_loss", C.c_float), ("rms_eps", C.c_float), ("attn_scale", C.c_float),
+                ("logit_scale", C.c_float),
+                ("dtype", C.c_int32), ("recompute", C.c_int32), ("flags", C.c_int32)]
+
+
+class t5_batch(C.Structure):
+    _fields_ = [("B", C.c_int32), ("Te", C.c_int32), ("Td", C.c_int32),
+                ("d_enc_tokens", C.c_void_p), ("d_enc_segment_ids", C.c_void_p),
+                ("d_dec_targets", C.c_void_p), ("d_dec_segment_ids", C.c_void_p)]
+
+
+EXPORTS = ["t5_create", "t5_destroy", "t5_last_error", "t5_param_count", "t5_param_tensors",
+           "t5_param_manifest", "t5_workspace_bytes", "t5_init_params", "t5_train_step_fwd_bwd",
+           "t5_encode", "t5_decode_logits", "t5_device_status", "t5_relpos_buckets", "t5_xent_zloss",
+           "t5_gemm"]
+
+_lib = None
+
+
+class T5Error(RuntimeError):
+    def __init__(self, code, msg=""):
+        super().__init__(f"{ERR_NAMES.get(code, code)}: {msg}")
+        self.code = code
+
+
+def lib():
+    """The loaded shared library (raises if it was not built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2203_17189_b200.build` "
+                               "(or __graft_entry__.build()) first; there is no fallback path")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
+        L.t5_create.argtypes = [C.POINTER(t5_config), C.POINTER(vp)]
+        L.t5_destroy.argtypes = [vp]
+        L.t5_last_error.argtypes = [vp]
+        L.t5_last_error.restype = C.c_char_p
+        L.t5_param_count.argtypes = [vp, C.POINTER(i64)]
+        L.t5_param_tensors.argtypes = [vp, C.POINTER(i32)]
+        L.t5_param_manifest.argtypes = [vp, i32, C.c_char_p, C.POINTER(i64), C.POINTER(i32 * 4), C.POINTER(i32)]
+        L.t5_workspace_bytes.argtypes = [vp, C.POINTER(i64)]
+        L.t5_init_params.argtypes = [vp, vp, C.c_uint64, f32, vp]
+        L.t5_train_step_fwd_bwd.argtypes = [vp, vp, C.POINTER(t5_batch), vp, vp, vp, i64, vp]
+        L.t5_encode.argtypes = [vp, vp, C.POINTER(t5_batch), vp, vp, i64, vp]
+        L.t5_decode_logits.argtypes = [vp, vp, C.POINTER(t5_batch), vp, vp, vp, i64, vp]
+        L.t5_device_status.argtypes = [vp, vp, vp]
+        L.t5_relpos_buckets.argtypes = [i32, i32, i32, i32, i32, vp, vp]
+        L.t5_xent_zloss.argtypes = [i32, vp, vp, i32, i32, f32, vp, vp, vp, vp]
+        L.t5_gemm.argtypes = [i32, i32, i32, i32, i32, f32, vp, i32, i32, vp, i32, i32, vp, i32, i32, i32, vp]
+        for n in EXPORTS:
+            if n != "t5_last_error":
+                getattr(L, n).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ptr(t):
+    return C.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _check(rc, h=None):
+    if rc != 0:
+        msg = lib().t5_last_error(h)
+        raise T5Error(rc, msg.decode() if msg else "")
+
+
+def make_config(dims, max_batch, max_enc_len, max_dec_len, dtype, *, z_loss=1e-4, rms_eps=1e-6,
+                attn_scale=1.0, logit_scale=None, rel_buckets=32, rel_max_distance=128,
+                recompute=0, flags=0):
+    """dims: mapping with arch, n_enc_layers, n_dec_layers, d_model, n_heads, d_kv, d_ff, vocab.
+    dtype: 'f32' or 'bf16'."""
+    c = t5_config()
+    c.abi_version = T5_ABI_VERSION
+    for k in ("arch", "n_enc_layers", "n_dec_layers", "d_model", "n_heads", "d_kv", "d_ff", "vocab"):
+        setattr(c, k, int(dims[k]))
+    c.rel_buckets, c.rel_max_distance = rel_buckets, rel_max_distance
+    c.max_batch, c.max_enc_len, c.max_dec_len = max_batch, max_enc_len, max_dec_len
+    c.z_loss, c.rms_eps, c.attn_scale = z_loss, rms_eps, attn_scale
+    c.logit_scale = float(dims["d_model"]) ** -0.5 if logit_scale is None else logit_scale
+    c.dtype = {"f32": 0, "bf16": 1}[dtype]
+    c.recompute, c.flags = recompute, flags
+    return c
+
+
+class Handle:
+    """Owns a t5_handle*; methods are the C calls with torch tensors as buffers."""
+
+    def __init__(self, cfg: t5_config):
+        self.cfg = cfg
+        self._h = C.c_void_p()
+        rc = lib().t5_create(C.byref(cfg), C.byref(self._h))
+        if rc != 0:
+            msg = lib().t5_last_error(None)
+            raise T5Error(rc, msg.decode() if msg else "")
+        self.torch_dtype = torch.float32 if cfg.dtype == 0 else torch.bfloat16
+
+    def close(self):
+        if self._h:
+            lib().t5_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def t5_param_count(self):
+        n = C.c_int64()
+        _check(lib().t5_param_count(self._h, C.byref(n)), self._h)
+        return n.value
+
+    def t5_param_manifest(self):
+        """List of (name, offset, shape)."""
+        n = C.c_int32()
+        _check(lib().t5_param_tensors(self._h, C.byref(n)), self._h)
+        out = []
+        for i in range(n.value):
+            name = C.create_string_buffer(64)
+            off = C.c_int64()
+            shape = (C.c_int32 * 4)()
+            nd = C.c_int32()
+            _check(lib().t5_param_manifest(self._h, i, name, C.byref(off), C.byref(shape), C.byref(nd)), self._h)
+            out.append((name.value.decode(), off.value, tuple(shape[:nd.value])))
+        return out
+
+    def t5_workspace_bytes(self):
+        n = C.c_int64()
+        _check(lib().t5_workspace_bytes(self._h, C.byref(n)), self._h)
+        return n.value
+
+    def t5_init_params(self, params, seed, stddev):
+        _check(lib().t5_init_params(self._h, _ptr(params), C.c_uint64(seed), stddev, _stream()), self._h)
+
+    def _batch(self, batch):
+        b = t5_batch()
+        dec = batch["dec_targets"]
+        b.B, b.Td = dec.shape
+        enc = batch.get("enc_tokens")
+        b.Te = 0 if enc is None else enc.shape[1]
+        b.d_enc_tokens = None if enc is None else enc.data_ptr()
+        es = batch.get("enc_segment_ids")
+        ds = batch.get("dec_segment_ids")
+        b.d_enc_segment_ids = None if es is None else es.data_ptr()
+        b.d_dec_targets = dec.data_ptr()
+        b.d_dec_segment_ids = None if ds is None else ds.data_ptr()
+        return b
+
+    def t5_train_step_fwd_bwd(self, params, batch, grads, loss4, workspace):
+        b = self._batch(batch)
+        _check(lib().t5_train_step_fwd_bwd(self._h, _ptr(params), C.byref(b), _ptr(grads), _ptr(loss4),
+                                           _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                           _stream()), self._h)
+
+    def t5_encode(self, params, batch, enc_out, workspace):
+        b = self._batch(batch)
+        _check(lib().t5_encode(self._h, _ptr(params), C.byref(b), _ptr(enc_out), _ptr(workspace),
+                               workspace.numel() * workspace.element_size(), _stream()), self._h)
+
+    def t5_decode_logits(self, params, batch, enc_out, logits, workspace):
+        b = self._batch(batch)
+        _check(lib().t5_decode_logits(self._h, _ptr(params), C.byref(b), _ptr(enc_out), _ptr(logits),
+                                      _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                      _stream()), self._h)
+
+    def t5_device_status(self, workspace):
+        _check(lib().t5_device_status(self._h, _ptr(workspace), _stream()), self._h)
+
+
+def t5_relpos_buckets(bidirectional, num_buckets, max_distance, rel_lo, out):
+    _check(lib().t5_relpos_buckets(int(bidirectional), num_buckets, max_distance, rel_lo, out.numel(),
+                                   _ptr(out), _stream()))
+
+
+def t5_xent_zloss(logits, targets, z_loss, W, sums, lse):
+    dtype = 0 if logits.dtype == torch.float32 else 1
+    n, v = logits.shape
+    _check(lib().t5_xent_zloss(dtype, _ptr(logits), _ptr(targets), n, v, z_loss, _ptr(W), _ptr(sums),
+                               _ptr(lse), _stream()))
+
+
+def t5_gemm(impl, M, N, K, alpha, A, lda, a_kmajor, B, ldb, b_kmajor, D, ldd, accumulate=False):
+    dtype = 0 if A.dtype == torch.float32 else 1
+    out_f32 = int(D.dtype == torch.float32)
+    _check(lib().t5_gemm(dtype, impl, M, N, K, alpha, _ptr(A), lda, int(a_kmajor), _ptr(B), ldb,
+                         int(b_kmajor), _ptr(D), ldd, out_f32, int(accumulate), _stream()))

@@ -1,0 +1,124 @@
+// Shared declarations of the GPU library: element types, the relative-position
+// bucket rule, and the launcher prototypes of every kernel family.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+typedef __nv_bfloat16 bf16;
+
+// dtype codes of the C ABI
+enum { DT_F32 = 0, DT_BF16 = 1 };
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+// ---------------------------------------------------------------------------
+// Relative-position bucket.  The closed form
+//   bucket = me + floor( log(n/me) / log(MD/me) * (nb - me) ), capped at nb-1,
+// is turned on the host into integer thresholds thr[q] = smallest n whose
+// floor(...) is >= q+1 (exact comparison of integer powers), so the device
+// only compares integers and both sides agree bit for bit.
+// ---------------------------------------------------------------------------
+#define T5_MAX_BUCKET_THR 128
+struct BucketSpec {
+  int bidirectional;
+  int nb;      // buckets available per direction (num_buckets/2 if bidirectional)
+  int me;      // nb/2: distances below this map to themselves
+  int n_thr;   // number of thresholds (= nb - me - 1 useful ones)
+  int thr[T5_MAX_BUCKET_THR];
+};
+
+__host__ __device__ inline int bucket_of(const BucketSpec& s, int rel) {
+  int off = 0, n;
+  if (s.bidirectional) {
+    if (rel > 0) off = s.nb;
+    n = rel < 0 ? -rel : rel;
+  } else {
+    n = rel < 0 ? -rel : 0;
+  }
+  if (n < s.me) return off + n;
+  int q = 0;
+  while (q < s.n_thr && n >= s.thr[q]) ++q;
+  return off + s.me + q;
+}
+
+// Builds the thresholds; returns false if the parameters are unsupported.
+bool build_bucket_spec(int bidirectional, int num_buckets, int max_distance, BucketSpec* out);
+
+// ---------------------------------------------------------------------------
+// Launchers.  `dtype` selects float / bf16 storage for "T" tensors; all
+// reductions and accumulators are float32.  Every launcher returns the
+// cudaError_t of its launch.
+// ---------------------------------------------------------------------------
+struct GemmArgs {
+  int M, N, K;
+  float alpha;
+  const void* A; int lda; int a_kmajor;   // A stored [M,K] if a_kmajor else [K,M]
+  const void* B; int ldb; int b_kmajor;   // B stored [N,K] if b_kmajor else [K,N]
+  void* D; int ldd; int out_f32;          // D[M,N]; float32 or operand dtype
+  const float* resid; int ldr;            // optional float32 addend (D may alias it)
+  int accumulate;                         // D += (float32 output only)
+};
+cudaError_t gemm_simt(int dtype, const GemmArgs& g, cudaStream_t st);
+// tcgen05 path: bf16 operands only.  `status` is a device int set non-zero if a
+// bounded wait inside the kernel ran out.
+cudaError_t gemm_tc(const GemmArgs& g, int* d_status, cudaStream_t st);
+bool gemm_tc_supported(const GemmArgs& g);
+
+struct AttnArgs {
+  // rows of Q/O/dQ/dO are (b*Tq + i), rows of K/V/dK/dV are (b*Tk + j);
+  // head h occupies columns [h*dk, (h+1)*dk) from each base pointer.
+  const void *Q, *K, *V;
+  void* O;
+  int ldq, ldk, ldv, ldo;
+  float* lse;               // [B,H,Tq]
+  int B, H, Tq, Tk, dk;
+  const int* code_q;        // [B,Tq]
+  const int* code_k;        // [B,Tk]
+  int causal;
+  const float* bias_delta;  // [H, Tq+Tk-1] indexed by (j - i + Tq - 1), or NULL
+  float scale;
+  // backward only
+  const void* dO; int lddo;
+  void *dQ, *dK, *dV; int lddq, lddk, lddv;
+  float* delta;             // [B,H,Tq] scratch: sum_d dO*O
+  float* dbias_delta;       // [H, Tq+Tk-1] float32, accumulated (+=), or NULL
+};
+cudaError_t attn_fwd_simt(int dtype, const AttnArgs& a, cudaStream_t st);
+cudaError_t attn_bwd_simt(int dtype, const AttnArgs& a, cudaStream_t st);
+
+// element-wise / row kernels
+cudaError_t launch_prep(const int* enc_tok, const int* enc_seg, const int* dec_tgt, const int* dec_seg,
+                        int B, int Te, int Td, int* enc_code, int* dec_code, int* dec_in,
+                        int* W_int, float* W_f, cudaStream_t st);
+cudaError_t launch_embed_gather(int dtype, const void* E, const int* tok, float* X, int n_tok, int d,
+                                cudaStream_t st);
+cudaError_t launch_embed_scatter_add(const int* tok, const float* dX, float* dE, int n_tok, int d,
+                                     cudaStream_t st);
+cudaError_t launch_rmsnorm_fwd(int dtype, const float* X, const void* g, void* Y, float* rstd,
+                               int rows, int d, float eps, cudaStream_t st);
+// dX_out = (dX_in ? dX_in : 0) + rmsnorm_bwd(dy); writes float32 dX_out and a T copy dXb (if non-NULL).
+// dy is float32 if dy_f32 else T.  dg (float32 [d]) is OVERWRITTEN; partial: scratch [n_part*d].
+cudaError_t launch_rmsnorm_bwd(int dtype, const void* dy, int dy_f32, const float* X, const float* rstd,
+                               const void* g, const float* dX_in, float* dX_out, void* dXb, float* dg,
+                               float* partial, int rows, int d, cudaStream_t st);
+int rmsnorm_bwd_parts(int rows);
+cudaError_t launch_geglu_fwd(int dtype, const void* h, void* hg, int rows, int F, cudaStream_t st);
+cudaError_t launch_geglu_bwd(int dtype, const void* dhg, const void* h, void* dh, int rows, int F,
+                             cudaStream_t st);
+cudaError_t launch_xent(int dtype, void* logits, const int* targets, int rows, int V, float z,
+                        const float* W, double* sums, float* lse, cudaStream_t st);
+cudaError_t launch_finalize_loss(const double* sums, const float* W, float* loss4, cudaStream_t st);
+cudaError_t launch_fill_normal(int dtype, void* p, int64_t n, int64_t flat_offset, uint64_t seed,
+                               float stddev, float mean, cudaStream_t st);
+cudaError_t launch_cast_f32_to(int dtype, const float* src, void* dst, int64_t n, cudaStream_t st);
+// bias tables
+cudaError_t launch_relbias_expand(int dtype, const BucketSpec& spec, const void* table, int H, int Tq,
+                                  int Tk, float* bias_delta, cudaStream_t st);
+cudaError_t launch_relbias_fold(const BucketSpec& spec, const float* dbias_delta, int H, int Tq, int Tk,
+                                int num_buckets, float* dtable, cudaStream_t st);
+cudaError_t launch_buckets(const BucketSpec& spec, int rel_lo, int n, int* out, cudaStream_t st);

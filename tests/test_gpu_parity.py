@@ -1,0 +1,253 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle
+on the same seeded inputs.
+
+Bars: bucket indices bit-exact; loss within 1e-3 relative; every gradient
+tensor at cosine >= 0.999 and max error <= 2e-2 of the tensor's largest
+magnitude with bfloat16 operands, <= 1e-4 in the float32 validation mode.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import t5_oracle as O
+from paper_2203_17189_b200 import binding as Bd
+from paper_2203_17189_b200 import workloads as WL
+from tests import parity as PR
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def to_dev(a):
+    return None if a is None else torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+
+
+def oracle_cfg(dims, **kw):
+    return O.T5Config(**{k: dims[k] for k in WL.MODEL_KEYS}, **kw)
+
+
+class Runner:
+    """One library handle plus its device buffers."""
+
+    def __init__(self, dims, B, Te, Td, dtype, flags=0, **cfg_kw):
+        self.dims = dims
+        self.cfg = Bd.make_config(dims, B, Te, Td, dtype, flags=flags, **cfg_kw)
+        self.h = Bd.Handle(self.cfg)
+        self.man = self.h.t5_param_manifest()
+        self.n = self.h.t5_param_count()
+        self.ws = torch.empty(self.h.t5_workspace_bytes(), dtype=torch.uint8, device=DEV)
+        self.grads = torch.empty(self.n, dtype=torch.float32, device=DEV)
+        self.loss4 = torch.zeros(4, dtype=torch.float32, device=DEV)
+        self.tdt = self.h.torch_dtype
+
+    def set_params(self, named):
+        flat = PR.pack_params(self.man, self.n, named)
+        self.params = torch.from_numpy(flat).to(DEV).to(self.tdt)
+        # what the device really holds (bf16-rounded), in the oracle's convention
+        return PR.unpack(self.man, self.params.float().cpu().numpy())
+
+    def step(self, batch):
+        self.batch = {k: to_dev(v) for k, v in batch.items()}
+        self.grads.fill_(float("nan"))
+        self.h.t5_train_step_fwd_bwd(self.params, self.batch, self.grads, self.loss4, self.ws)
+        torch.cuda.synchronize()
+        self.h.t5_device_status(self.ws)
+        return self.loss4.cpu().numpy().astype(np.float64), self.grads.cpu().numpy()
+
+
+def check_step(dims, batch, dtype, flags=0, seed=11, stddev=0.05, tol=None, table_out=None):
+    B, Td = batch["dec_targets"].shape
+    Te = 0 if batch["enc_tokens"] is None else batch["enc_tokens"].shape[1]
+    r = Runner(dims, B, Te, Td, dtype, flags=flags)
+    shapes = PR.oracle_shapes_from_manifest(r.man)
+    named = WL.make_params(shapes, seed, stddev=stddev, scale_jitter=0.05)
+    named = r.set_params(named)
+    loss4, grads = r.step(batch)
+    ocfg = oracle_cfg(dims)
+    oloss, ograds = O.t5_train_step(ocfg, named, batch["enc_tokens"], batch["enc_segment_ids"],
+                                    batch["dec_targets"], batch["dec_segment_ids"], dtype=np.float64)
+    assert np.isfinite(grads).all()
+    assert loss4[3] == oloss[3]
+    assert abs(loss4[0] - oloss[0]) <= 1e-3 * abs(oloss[0]), (loss4, oloss)
+    assert abs(loss4[1] - oloss[1]) <= 1e-3 * abs(oloss[1])
+    assert abs(loss4[2] - oloss[2]) <= 2e-3 * abs(oloss[2]) + 1e-7
+    wc, wr, table = PR.compare_grads(r.man, grads, ograds)
+    if table_out is not None:
+        table_out.update(table)
+    cos_min, rel_max = tol if tol else ((0.999999, 1e-4) if dtype == "f32" else (0.999, 2e-2))
+    bad = {k: v for k, v in table.items() if v[0] < cos_min or v[1] > rel_max}
+    assert not bad, bad
+    return r, named, loss4, grads
+
+
+# ------------------------------------------------------------------ single operations
+@pytest.mark.parametrize("bidir", [True, False])
+def test_bucket_indices_bit_exact(bidir):
+    lo, n = -2047, 4095
+    out = torch.empty(n, dtype=torch.int32, device=DEV)
+    Bd.t5_relpos_buckets(bidir, 32, 128, lo, out)
+    got = out.cpu().numpy()
+    want = np.array([O.relative_position_bucket(lo + i, bidir, 32, 128) for i in range(n)], dtype=np.int32)
+    assert np.array_equal(got, want)
+
+
+def test_bucket_other_parameters_bit_exact():
+    for nb, md in ((16, 64), (64, 256), (32, 20)):
+        out = torch.empty(1201, dtype=torch.int32, device=DEV)
+        for bidir in (True, False):
+            Bd.t5_relpos_buckets(bidir, nb, md, -600, out)
+            want = [O.relative_position_bucket(-600 + i, bidir, nb, md) for i in range(1201)]
+            assert out.cpu().tolist() == want
+
+
+@pytest.mark.parametrize("dtype,rows,V", [("f32", 37, 512), ("bf16", 300, 32128), ("f32", 5, 40)])
+def test_xent_zloss_rows(dtype, rows, V):
+    rng = np.random.default_rng(5)
+    logits = (rng.standard_normal((rows, V)) * 3).astype(np.float32)
+    tgt = rng.integers(1, V, size=rows).astype(np.int32)
+    tgt[rows // 3] = 0
+    tgt[rows - 1] = 0
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    dl = torch.from_numpy(logits).to(DEV).to(tdt)
+    held = dl.float().cpu().numpy().astype(np.float64)
+    W = float((tgt != 0).sum())
+    dW = torch.tensor([W], dtype=torch.float32, device=DEV)
+    sums = torch.zeros(2, dtype=torch.float64, device=DEV)
+    lse = torch.empty(rows, dtype=torch.float32, device=DEV)
+    Bd.t5_xent_zloss(dl, to_dev(tgt), 1e-4, dW, sums, lse)
+    torch.cuda.synchronize()
+    w = (tgt != 0).astype(np.float64)
+    ce_t, zl_t, olse, prob = O.xent_zloss_row(held, tgt, w, 1e-4)
+    want = prob * (1 + 2e-4 * olse)[:, None]
+    want[np.arange(rows), tgt] -= 1
+    want *= (w / W)[:, None]
+    got = dl.float().cpu().numpy()
+    assert np.allclose(lse.cpu().numpy(), olse, rtol=2e-6, atol=2e-6)
+    s = sums.cpu().numpy()
+    assert abs(s[0] - (w * ce_t).sum()) <= 1e-5 * abs((w * ce_t).sum())
+    assert abs(s[1] - (w * zl_t).sum()) <= 1e-5 * abs((w * zl_t).sum())
+    tol = 1e-5 if dtype == "f32" else 1e-2
+    assert np.abs(got - want).max() <= tol * np.abs(want).max()
+    assert np.all(got[tgt == 0] == 0)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("ak,bk", [(1, 1), (1, 0), (0, 0), (0, 1)])
+def test_gemm_simt_against_matmul(dtype, ak, bk):
+    M, N, K = 150, 203, 77
+    rng = np.random.default_rng(1)
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    A = torch.from_numpy(rng.standard_normal((M, K)).astype(np.float32)).to(DEV).to(tdt)
+    Bm = torch.from_numpy(rng.standard_normal((N, K)).astype(np.float32)).to(DEV).to(tdt)
+    ref = A.double().cpu().numpy() @ Bm.double().cpu().numpy().T
+    As = A if ak else A.t().contiguous()
+    Bs = Bm if bk else Bm.t().contiguous()
+    D = torch.zeros(M, N, dtype=torch.float32, device=DEV)
+    Bd.t5_gemm(0, M, N, K, 0.5, As, As.stride(0), ak, Bs, Bs.stride(0), bk, D, N)
+    Bd.t5_gemm(0, M, N, K, 0.5, As, As.stride(0), ak, Bs, Bs.stride(0), bk, D, N, accumulate=True)
+    torch.cuda.synchronize()
+    assert np.abs(D.cpu().numpy() - ref).max() <= 1e-4 * np.abs(ref).max()
+
+
+# ------------------------------------------------------------------ whole step
+def test_step_tiny_config_fp32():
+    """The smallest workload in full: float32 validation mode."""
+    dims = WL.model_dims("tiny")
+    batch = WL.make_batch("tiny")
+    check_step(dims, batch, "f32", stddev=0.02)
+    check_step(dims, batch, "f32", stddev=0.08, seed=3)
+
+
+def test_step_tiny_config_bf16_simt():
+    dims = WL.model_dims("tiny")
+    batch = WL.make_batch("tiny")
+    check_step(dims, batch, "bf16", flags=1, stddev=0.05)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_step_padded_ragged_lengths(dtype):
+    """Lengths that are not multiples of any tile (Te=75, Td=21), trailing padding, d_kv=64, I != d."""
+    dims = WL.model_dims("small", n_enc_layers=2, n_dec_layers=2, vocab=1000, d_model=192, n_heads=2,
+                         d_ff=320, enc_len=75, dec_len=21, batch=3, padding=0.2)
+    batch = WL.make_batch(dims, seed=7)
+    check_step(dims, batch, dtype)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_step_packed_segments(dtype):
+    dims = WL.model_dims("base", n_enc_layers=1, n_dec_layers=2, vocab=2000, d_model=128, n_heads=4,
+                         d_kv=32, d_ff=256, enc_len=96, dec_len=40, batch=3)
+    batch = WL.make_batch(dims, seed=8)
+    assert batch["enc_segment_ids"].max() >= 2
+    check_step(dims, batch, dtype)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_step_decoder_only_packed(dtype):
+    dims = WL.model_dims("declm", n_dec_layers=2, vocab=2000, d_model=256, n_heads=2, d_kv=128, d_ff=384,
+                         dec_len=150, batch=2)
+    batch = WL.make_batch(dims, seed=9)
+    check_step(dims, batch, dtype)
+
+
+def test_all_padding_gives_zero():
+    dims = WL.model_dims("tiny")
+    batch = WL.make_batch("tiny")
+    batch["dec_targets"][:] = 0
+    r = Runner(dims, 4, 64, 32, "f32")
+    r.set_params(WL.make_params(PR.oracle_shapes_from_manifest(r.man), 1))
+    loss4, grads = r.step(batch)
+    assert np.all(loss4 == 0) and np.all(grads == 0)
+
+
+def test_encode_and_decode_logits_match_oracle():
+    dims = WL.model_dims("tiny")
+    batch = WL.make_batch("tiny")
+    batch["enc_tokens"][1, 50:] = 0
+    batch["dec_targets"][2, 20:] = 0
+    r = Runner(dims, 4, 64, 32, "f32")
+    named = r.set_params(WL.make_params(PR.oracle_shapes_from_manifest(r.man), 2, stddev=0.05))
+    dev_batch = {k: to_dev(v) for k, v in batch.items()}
+    enc_out = torch.empty(4, 64, 128, dtype=torch.float32, device=DEV)
+    logits = torch.empty(4, 32, 512, dtype=torch.float32, device=DEV)
+    r.h.t5_encode(r.params, dev_batch, enc_out, r.ws)
+    r.h.t5_decode_logits(r.params, dev_batch, enc_out, logits, r.ws)
+    torch.cuda.synchronize()
+    ocfg = oracle_cfg(dims)
+    oe = O.t5_encode(ocfg, named, batch["enc_tokens"], None)
+    ol = O.t5_decode_logits(ocfg, named, oe, batch["enc_tokens"], None, batch["dec_targets"], None)
+    valid = batch["enc_tokens"] != 0      # padding queries are outside the contract
+    assert np.abs(enc_out.cpu().numpy() - oe)[valid].max() <= 1e-4 * np.abs(oe).max()
+    vd = batch["dec_targets"] != 0
+    assert np.abs(logits.cpu().numpy() - ol)[vd].max() <= 1e-4 * np.abs(ol).max()
+
+
+def test_argument_errors_on_device():
+    dims = WL.model_dims("tiny")
+    r = Runner(dims, 4, 64, 32, "f32")
+    r.set_params(WL.make_params(PR.oracle_shapes_from_manifest(r.man), 1))
+    batch = WL.make_batch("tiny", batch=6)           # more rows than max_batch
+    with pytest.raises(Bd.T5Error) as e:
+        r.step(batch)
+    assert e.value.code == -3
+    small_ws = r.ws[:1024]
+    with pytest.raises(Bd.T5Error) as e:
+        r.h.t5_train_step_fwd_bwd(r.params, {k: to_dev(v) for k, v in WL.make_batch("tiny").items()}, r.grads,
+                                  r.loss4, small_ws)
+    assert e.value.code == -5
+
+
+def test_init_params_statistics():
+    dims = WL.model_dims("tiny")
+    r = Runner(dims, 4, 64, 32, "f32")
+    p = torch.empty(r.n, dtype=torch.float32, device=DEV)
+    r.h.t5_init_params(p, 42, 0.02)
+    p2 = torch.empty(r.n, dtype=torch.float32, device=DEV)
+    r.h.t5_init_params(p2, 42, 0.02)
+    torch.cuda.synchronize()
+    assert torch.equal(p, p2)
+    named = PR.unpack(r.man, p.cpu().numpy())
+    assert np.all(named["enc.L0.attn.norm"] == 1.0)
+    e = named["token_embed"]
+    assert abs(e.mean()) < 1e-3 and abs(e.std() - 0.02) < 5e-4
+    assert abs(np.mean(e ** 4) / np.mean(e ** 2) ** 2 - 3.0) < 0.15     # Gaussian kurtosis
