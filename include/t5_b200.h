@@ -150,6 +150,18 @@ T5_API int t5_decode_logits(t5_handle* h, const void* d_params, const t5_batch* 
  * Returns T5_OK or T5_ERR_DEVICE_TIMEOUT. */
 T5_API int t5_device_status(t5_handle* h, const void* d_workspace, void* stream);
 
+/* Measurement aids (no counterpart in the paper).  With profiling enabled every
+ * kernel launch of the following calls is bracketed by a CUDA event pair on the
+ * caller's stream.  t5_profile_read() waits for those events, returns per kernel
+ * family the summed device time (ms), the algorithmic FLOPs of its GEMMs and
+ * the number of kernels, then clears the record.  Families: 0 GEMM,
+ * 1 attention forward, 2 attention backward, 3 RMSNorm, 4 gated GELU,
+ * 5 cross-entropy, 6 embedding, 7 other.  t5_launch_count(): kernels launched
+ * by the most recent step/encode/decode call on this handle. */
+T5_API int t5_profile_enable(t5_handle* h, int32_t on);
+T5_API int t5_profile_read(t5_handle* h, double ms[8], double flops[8], int64_t launches[8]);
+T5_API int t5_launch_count(const t5_handle* h, int64_t* n);
+
 /* ---- single operations of the path, exported for element-wise parity tests ---- */
 
 /* Relative-position bucket (closed form, exact integer thresholds):

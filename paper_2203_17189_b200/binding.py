@@ -40,7 +40,8 @@ class t5_batch(C.Structure):
 
 EXPORTS = ["t5_create", "t5_destroy", "t5_last_error", "t5_param_count", "t5_param_tensors",
            "t5_param_manifest", "t5_workspace_bytes", "t5_init_params", "t5_train_step_fwd_bwd",
-           "t5_encode", "t5_decode_logits", "t5_device_status", "t5_relpos_buckets", "t5_xent_zloss",
+           "t5_encode", "t5_decode_logits", "t5_device_status", "t5_profile_enable", "t5_profile_read",
+           "t5_launch_count", "t5_relpos_buckets", "t5_xent_zloss",
            "t5_gemm"]
 
 _lib = None
@@ -74,6 +75,10 @@ def lib():
         L.t5_encode.argtypes = [vp, vp, C.POINTER(t5_batch), vp, vp, i64, vp]
         L.t5_decode_logits.argtypes = [vp, vp, C.POINTER(t5_batch), vp, vp, vp, i64, vp]
         L.t5_device_status.argtypes = [vp, vp, vp]
+        L.t5_profile_enable.argtypes = [vp, i32]
+        L.t5_profile_read.argtypes = [vp, C.POINTER(C.c_double * 8), C.POINTER(C.c_double * 8),
+                                      C.POINTER(i64 * 8)]
+        L.t5_launch_count.argtypes = [vp, C.POINTER(i64)]
         L.t5_relpos_buckets.argtypes = [i32, i32, i32, i32, i32, vp, vp]
         L.t5_xent_zloss.argtypes = [i32, vp, vp, i32, i32, f32, vp, vp, vp, vp]
         L.t5_gemm.argtypes = [i32, i32, i32, i32, i32, f32, vp, i32, i32, vp, i32, i32, vp, i32, i32, i32, vp]
@@ -196,6 +201,21 @@ class Handle:
         _check(lib().t5_decode_logits(self._h, _ptr(params), C.byref(b), _ptr(enc_out), _ptr(logits),
                                       _ptr(workspace), workspace.numel() * workspace.element_size(),
                                       _stream()), self._h)
+
+    def t5_profile_enable(self, on):
+        _check(lib().t5_profile_enable(self._h, int(on)), self._h)
+
+    def t5_profile_read(self):
+        """{family: (ms, flops, launches)}"""
+        ms, fl, ln = (C.c_double * 8)(), (C.c_double * 8)(), (C.c_int64 * 8)()
+        _check(lib().t5_profile_read(self._h, C.byref(ms), C.byref(fl), C.byref(ln)), self._h)
+        names = ["gemm", "attn_fwd", "attn_bwd", "rmsnorm", "geglu", "xent", "embed", "other"]
+        return {n: (ms[i], fl[i], ln[i]) for i, n in enumerate(names)}
+
+    def t5_launch_count(self):
+        n = C.c_int64()
+        _check(lib().t5_launch_count(self._h, C.byref(n)), self._h)
+        return n.value
 
     def t5_device_status(self, workspace):
         _check(lib().t5_device_status(self._h, _ptr(workspace), _stream()), self._h)

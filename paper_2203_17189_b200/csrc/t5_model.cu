@@ -59,6 +59,13 @@ struct t5_handle {
   std::vector<DecLayerP> dec;
   BucketSpec spec_enc, spec_dec;
   std::string err;
+  // opt-in per-kernel-family timing (CUDA events around each launch) and launch counting
+  bool prof_on = false;
+  std::vector<cudaEvent_t> prof_events;      // pairs: start, stop
+  std::vector<int> prof_cat;                 // category of each pair in use
+  double prof_flops[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  int64_t prof_launches[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  int64_t launches_last_call = 0;
 };
 
 namespace {
@@ -238,8 +245,36 @@ struct Ctx {
   int B, Te, Td;
   cudaError_t err;
   const char* where;
+  int64_t launches;
 };
 
+enum { CAT_GEMM = 0, CAT_ATTN_FWD, CAT_ATTN_BWD, CAT_NORM, CAT_GEGLU, CAT_XENT, CAT_EMBED, CAT_MISC };
+
+// Records a start/stop event pair around the launches made while it is alive (profiling mode only).
+struct ProfScope {
+  Ctx& cx;
+  int idx = -1;
+  ProfScope(Ctx& c, int cat, double flops, int n_kernels) : cx(c) {
+    cx.launches += n_kernels;
+    t5_handle* h = cx.h;
+    if (!h->prof_on || cx.err != cudaSuccess) return;
+    idx = (int)h->prof_cat.size();
+    while ((int)h->prof_events.size() < 2 * (idx + 1)) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) { idx = -1; return; }
+      h->prof_events.push_back(e);
+    }
+    h->prof_cat.push_back(cat);
+    h->prof_flops[cat] += flops;
+    h->prof_launches[cat] += n_kernels;
+    cudaEventRecord(h->prof_events[2 * idx], cx.st);
+  }
+  ~ProfScope() {
+    if (idx >= 0) cudaEventRecord(cx.h->prof_events[2 * idx + 1], cx.st);
+  }
+};
+
+// CK(call, what): plain runtime call.  CKL(cat, n, call, what): a launch of n kernels of family cat.
 #define CK(call, what)                                            \
   do {                                                            \
     if (cx.err == cudaSuccess) {                                  \
@@ -247,9 +282,19 @@ struct Ctx {
       if (e_ != cudaSuccess) { cx.err = e_; cx.where = what; }    \
     }                                                             \
   } while (0)
+#define CKL(cat, n, call, what)                                   \
+  do {                                                            \
+    if (cx.err == cudaSuccess) {                                  \
+      ProfScope ps_(cx, cat, 0.0, n);                             \
+      cudaError_t e_ = (call);                                    \
+      if (e_ != cudaSuccess) { cx.err = e_; cx.where = what; }    \
+    }                                                             \
+  } while (0)
 
 void gemm(Ctx& cx, const GemmArgs& g, const char* what) {
   int dt = cx.h->cfg.dtype;
+  if (cx.err != cudaSuccess) return;
+  ProfScope ps(cx, CAT_GEMM, 2.0 * g.M * g.N * g.K, 1);
   if (dt == DT_BF16 && !(cx.h->cfg.flags & 1) && gemm_tc_supported(g)) {
     CK(gemm_tc(g, cx.w->status, cx.st), what);
   } else {
@@ -319,7 +364,7 @@ void attn_forward(Ctx& cx, const AttnP& p, const AttnWs& a, float* x_out, const 
   const t5_config& c = cx.h->cfg;
   int d = c.d_model, I = c.n_heads * c.d_kv, dt = c.dtype;
   bool cross = kv_src != nullptr;
-  CK(launch_rmsnorm_fwd(dt, a.x, pptr(cx.h, cx.params, p.norm), a.y, a.rstd, (int)gm.Nq, d, c.rms_eps, cx.st),
+  CKL(CAT_NORM, 1, launch_rmsnorm_fwd(dt, a.x, pptr(cx.h, cx.params, p.norm), a.y, a.rstd, (int)gm.Nq, d, c.rms_eps, cx.st),
      "rmsnorm_fwd");
   if (!cross) {
     proj_fwd(cx, a.y, d, p.q, (int)gm.Nq, 3 * I, d, a.q, 3 * I, 1.f, nullptr, "qkv proj");
@@ -329,7 +374,7 @@ void attn_forward(Ctx& cx, const AttnP& p, const AttnWs& a, float* x_out, const 
   }
   AttnArgs t;
   attn_args(cx, a, gm, cross, &t);
-  CK(attn_fwd_simt(dt, t, cx.st), "attn_fwd");
+  CKL(CAT_ATTN_FWD, 1, attn_fwd_simt(dt, t, cx.st), "attn_fwd");
   proj_fwd(cx, a.ctx, I, p.o, (int)gm.Nq, d, I, x_out, d, 1.f, a.x, "o proj");
 }
 
@@ -353,7 +398,7 @@ void attn_backward(Ctx& cx, const AttnP& p, const AttnWs& a, float* dX, void* dX
     t.dQ = w.dqkv; t.dK = eoff(cx.h, w.dqkv, I); t.dV = eoff(cx.h, w.dqkv, 2 * I);
     t.lddq = t.lddk = t.lddv = 3 * I;
   }
-  CK(attn_bwd_simt(dt, t, cx.st), "attn_bwd");
+  CKL(CAT_ATTN_BWD, 3, attn_bwd_simt(dt, t, cx.st), "attn_bwd");
   if (!cross) {
     proj_wgrad(cx, w.dqkv, 3 * I, a.y, d, p.q, Nq, 3 * I, d, 1.f, "wgrad qkv");
     proj_dgrad(cx, w.dqkv, 3 * I, p.q, Nq, 3 * I, d, w.dy, d, 1.f, 0, 0, "dgrad qkv");
@@ -363,7 +408,7 @@ void attn_backward(Ctx& cx, const AttnP& p, const AttnWs& a, float* dX, void* dX
     proj_wgrad(cx, w.dkv, 2 * I, kv_src, d, p.k, Nk, 2 * I, d, 1.f, "wgrad kv");
     proj_dgrad(cx, w.dkv, 2 * I, p.k, Nk, 2 * I, d, dY32, d, 1.f, 1, dY_accumulate, "dgrad kv");
   }
-  CK(launch_rmsnorm_bwd(dt, w.dy, 0, a.x, a.rstd, pptr(cx.h, cx.params, p.norm), dX, dX, dXb, cx.grads + p.norm,
+  CKL(CAT_NORM, 2, launch_rmsnorm_bwd(dt, w.dy, 0, a.x, a.rstd, pptr(cx.h, cx.params, p.norm), dX, dX, dXb, cx.grads + p.norm,
                         w.norm_partial, Nq, d, cx.st),
      "rmsnorm_bwd");
 }
@@ -371,10 +416,10 @@ void attn_backward(Ctx& cx, const AttnP& p, const AttnWs& a, float* dX, void* dX
 void ffn_forward(Ctx& cx, const FfnP& p, const FfnWs& f, float* x_out, int64_t N) {
   const t5_config& c = cx.h->cfg;
   int d = c.d_model, F = c.d_ff, dt = c.dtype;
-  CK(launch_rmsnorm_fwd(dt, f.x, pptr(cx.h, cx.params, p.norm), f.y, f.rstd, (int)N, d, c.rms_eps, cx.st),
+  CKL(CAT_NORM, 1, launch_rmsnorm_fwd(dt, f.x, pptr(cx.h, cx.params, p.norm), f.y, f.rstd, (int)N, d, c.rms_eps, cx.st),
      "rmsnorm_fwd");
   proj_fwd(cx, f.y, d, p.wi0, (int)N, 2 * F, d, f.h, 2 * F, 1.f, nullptr, "wi proj");
-  CK(launch_geglu_fwd(dt, f.h, f.hg, (int)N, F, cx.st), "geglu_fwd");
+  CKL(CAT_GEGLU, 1, launch_geglu_fwd(dt, f.h, f.hg, (int)N, F, cx.st), "geglu_fwd");
   proj_fwd(cx, f.hg, F, p.wo, (int)N, d, F, x_out, d, 1.f, f.x, "wo proj");
 }
 
@@ -384,10 +429,10 @@ void ffn_backward(Ctx& cx, const FfnP& p, const FfnWs& f, float* dX, void* dXb, 
   int d = c.d_model, F = c.d_ff, dt = c.dtype, n = (int)N;
   proj_wgrad(cx, dXb, d, f.hg, F, p.wo, n, d, F, 1.f, "wgrad ffn.wo");
   proj_dgrad(cx, dXb, d, p.wo, n, d, F, w.dhg, F, 1.f, 0, 0, "dgrad ffn.wo");
-  CK(launch_geglu_bwd(dt, w.dhg, f.h, w.dh, n, F, cx.st), "geglu_bwd");
+  CKL(CAT_GEGLU, 1, launch_geglu_bwd(dt, w.dhg, f.h, w.dh, n, F, cx.st), "geglu_bwd");
   proj_wgrad(cx, w.dh, 2 * F, f.y, d, p.wi0, n, 2 * F, d, 1.f, "wgrad ffn.wi");
   proj_dgrad(cx, w.dh, 2 * F, p.wi0, n, 2 * F, d, w.dy, d, 1.f, 0, 0, "dgrad ffn.wi");
-  CK(launch_rmsnorm_bwd(dt, w.dy, 0, f.x, f.rstd, pptr(cx.h, cx.params, p.norm), dX, dX, dXb, cx.grads + p.norm,
+  CKL(CAT_NORM, 2, launch_rmsnorm_bwd(dt, w.dy, 0, f.x, f.rstd, pptr(cx.h, cx.params, p.norm), dX, dX, dXb, cx.grads + p.norm,
                         w.norm_partial, n, d, cx.st),
      "rmsnorm_bwd");
 }
@@ -415,14 +460,14 @@ void run_prep(Ctx& cx, const t5_batch* b) {
   Workspace& w = *cx.w;
   const t5_config& c = cx.h->cfg;
   CK(cudaMemsetAsync(w.status, 0, 4, cx.st), "memset status");
-  CK(launch_prep(c.arch == 0 ? b->d_enc_tokens : nullptr, b->d_enc_segment_ids, b->d_dec_targets,
+  CKL(CAT_MISC, 2, launch_prep(c.arch == 0 ? b->d_enc_tokens : nullptr, b->d_enc_segment_ids, b->d_dec_targets,
                  b->d_dec_segment_ids, cx.B, cx.Te, cx.Td, w.enc_code, w.dec_code, w.dec_in, w.W_int, w.W_f, cx.st),
      "prep");
   if (c.arch == 0 && cx.Te > 0)
-    CK(launch_relbias_expand(c.dtype, cx.h->spec_enc, pptr(cx.h, cx.params, cx.h->enc_relbias), c.n_heads, cx.Te,
+    CKL(CAT_MISC, 1, launch_relbias_expand(c.dtype, cx.h->spec_enc, pptr(cx.h, cx.params, cx.h->enc_relbias), c.n_heads, cx.Te,
                              cx.Te, w.bias_enc, cx.st),
        "relbias_expand enc");
-  CK(launch_relbias_expand(c.dtype, cx.h->spec_dec, pptr(cx.h, cx.params, cx.h->dec_relbias), c.n_heads, cx.Td,
+  CKL(CAT_MISC, 1, launch_relbias_expand(c.dtype, cx.h->spec_dec, pptr(cx.h, cx.params, cx.h->dec_relbias), c.n_heads, cx.Td,
                            cx.Td, w.bias_dec, cx.st),
      "relbias_expand dec");
 }
@@ -433,7 +478,7 @@ void encoder_forward(Ctx& cx, const t5_batch* b) {
   int L = c.n_enc_layers, d = c.d_model;
   int64_t Ne = (int64_t)cx.B * cx.Te;
   float* x0 = L > 0 ? w.enc_attn[0].x : w.enc_x_final;
-  CK(launch_embed_gather(c.dtype, pptr(cx.h, cx.params, cx.h->token_embed), b->d_enc_tokens, x0, (int)Ne, d, cx.st),
+  CKL(CAT_EMBED, 1, launch_embed_gather(c.dtype, pptr(cx.h, cx.params, cx.h->token_embed), b->d_enc_tokens, x0, (int)Ne, d, cx.st),
      "embed enc");
   AttnGeom g = enc_geom(cx);
   for (int l = 0; l < L; ++l) {
@@ -441,7 +486,7 @@ void encoder_forward(Ctx& cx, const t5_batch* b) {
     float* x_next = l + 1 < L ? w.enc_attn[l + 1].x : w.enc_x_final;
     ffn_forward(cx, cx.h->enc[l].ffn, w.enc_ffn[l], x_next, Ne);
   }
-  CK(launch_rmsnorm_fwd(c.dtype, w.enc_x_final, pptr(cx.h, cx.params, cx.h->enc_final_norm), w.enc_out,
+  CKL(CAT_NORM, 1, launch_rmsnorm_fwd(c.dtype, w.enc_x_final, pptr(cx.h, cx.params, cx.h->enc_final_norm), w.enc_out,
                         w.enc_rstd_f, (int)Ne, d, c.rms_eps, cx.st),
      "enc final norm");
 }
@@ -453,7 +498,7 @@ void decoder_forward(Ctx& cx, const void* enc_y, void* logits_out) {
   int L = c.n_dec_layers, d = c.d_model;
   int64_t Nd = (int64_t)cx.B * cx.Td;
   float* x0 = L > 0 ? w.dec_self[0].x : w.dec_x_final;
-  CK(launch_embed_gather(c.dtype, pptr(cx.h, cx.params, cx.h->token_embed), w.dec_in, x0, (int)Nd, d, cx.st),
+  CKL(CAT_EMBED, 1, launch_embed_gather(c.dtype, pptr(cx.h, cx.params, cx.h->token_embed), w.dec_in, x0, (int)Nd, d, cx.st),
      "embed dec");
   AttnGeom gs = self_geom(cx), gc = cross_geom(cx);
   bool encdec = c.arch == 0;
@@ -464,7 +509,7 @@ void decoder_forward(Ctx& cx, const void* enc_y, void* logits_out) {
     float* x_next = l + 1 < L ? w.dec_self[l + 1].x : w.dec_x_final;
     ffn_forward(cx, cx.h->dec[l].ffn, w.dec_ffn[l], x_next, Nd);
   }
-  CK(launch_rmsnorm_fwd(c.dtype, w.dec_x_final, pptr(cx.h, cx.params, cx.h->dec_final_norm), w.dec_z, w.dec_rstd_f,
+  CKL(CAT_NORM, 1, launch_rmsnorm_fwd(c.dtype, w.dec_x_final, pptr(cx.h, cx.params, cx.h->dec_final_norm), w.dec_z, w.dec_rstd_f,
                         (int)Nd, d, c.rms_eps, cx.st),
      "dec final norm");
   proj_fwd(cx, w.dec_z, d, cx.h->token_embed, (int)Nd, c.vocab, d, logits_out, c.vocab, c.logit_scale, nullptr,
@@ -484,7 +529,7 @@ void backward(Ctx& cx, const t5_batch* b) {
   // tied embedding: dE = logit_scale dlogits^T Z (overwrites), dZ = logit_scale dlogits E
   proj_wgrad(cx, w.logits, V, w.dec_z, d, cx.h->token_embed, (int)Nd, V, d, c.logit_scale, "wgrad logits");
   proj_dgrad(cx, w.logits, V, cx.h->token_embed, (int)Nd, V, d, w.dy, d, c.logit_scale, 0, 0, "dgrad logits");
-  CK(launch_rmsnorm_bwd(dt, w.dy, 0, w.dec_x_final, w.dec_rstd_f, pptr(cx.h, cx.params, cx.h->dec_final_norm),
+  CKL(CAT_NORM, 2, launch_rmsnorm_bwd(dt, w.dy, 0, w.dec_x_final, w.dec_rstd_f, pptr(cx.h, cx.params, cx.h->dec_final_norm),
                         nullptr, w.dX_dec, w.dXb_dec, cx.grads + cx.h->dec_final_norm, w.norm_partial, (int)Nd, d,
                         cx.st),
      "dec final norm bwd");
@@ -499,13 +544,13 @@ void backward(Ctx& cx, const t5_batch* b) {
     }
     attn_backward(cx, cx.h->dec[l].self, w.dec_self[l], w.dX_dec, w.dXb_dec, gs, nullptr, nullptr, 0);
   }
-  CK(launch_embed_scatter_add(w.dec_in, w.dX_dec, cx.grads + cx.h->token_embed, (int)Nd, d, cx.st),
+  CKL(CAT_EMBED, 1, launch_embed_scatter_add(w.dec_in, w.dX_dec, cx.grads + cx.h->token_embed, (int)Nd, d, cx.st),
      "embed scatter dec");
-  CK(launch_relbias_fold(cx.h->spec_dec, w.dbias_dec, H, cx.Td, cx.Td, c.rel_buckets, cx.grads + cx.h->dec_relbias,
+  CKL(CAT_MISC, 1, launch_relbias_fold(cx.h->spec_dec, w.dbias_dec, H, cx.Td, cx.Td, c.rel_buckets, cx.grads + cx.h->dec_relbias,
                          cx.st),
      "relbias fold dec");
   if (!encdec) return;
-  CK(launch_rmsnorm_bwd(dt, w.dY32, 1, w.enc_x_final, w.enc_rstd_f, pptr(cx.h, cx.params, cx.h->enc_final_norm),
+  CKL(CAT_NORM, 2, launch_rmsnorm_bwd(dt, w.dY32, 1, w.enc_x_final, w.enc_rstd_f, pptr(cx.h, cx.params, cx.h->enc_final_norm),
                         nullptr, w.dX_enc, w.dXb_enc, cx.grads + cx.h->enc_final_norm, w.norm_partial, (int)Ne, d,
                         cx.st),
      "enc final norm bwd");
@@ -514,9 +559,9 @@ void backward(Ctx& cx, const t5_batch* b) {
     ffn_backward(cx, cx.h->enc[l].ffn, w.enc_ffn[l], w.dX_enc, w.dXb_enc, Ne);
     attn_backward(cx, cx.h->enc[l].attn, w.enc_attn[l], w.dX_enc, w.dXb_enc, ge, nullptr, nullptr, 0);
   }
-  CK(launch_embed_scatter_add(b->d_enc_tokens, w.dX_enc, cx.grads + cx.h->token_embed, (int)Ne, d, cx.st),
+  CKL(CAT_EMBED, 1, launch_embed_scatter_add(b->d_enc_tokens, w.dX_enc, cx.grads + cx.h->token_embed, (int)Ne, d, cx.st),
      "embed scatter enc");
-  CK(launch_relbias_fold(cx.h->spec_enc, w.dbias_enc, H, cx.Te, cx.Te, c.rel_buckets, cx.grads + cx.h->enc_relbias,
+  CKL(CAT_MISC, 1, launch_relbias_fold(cx.h->spec_enc, w.dbias_enc, H, cx.Te, cx.Te, c.rel_buckets, cx.grads + cx.h->enc_relbias,
                          cx.st),
      "relbias fold enc");
 }
@@ -542,11 +587,12 @@ int begin_call(t5_handle* h, const void* params, const t5_batch* b, void* ws, in
     return fail(h, T5_ERR_WORKSPACE, "workspace of %lld bytes given, %lld needed", (long long)ws_bytes,
                 (long long)w->bytes);
   cx->h = h; cx->params = params; cx->grads = nullptr; cx->st = (cudaStream_t)stream; cx->w = w;
-  cx->B = b->B; cx->Te = Te; cx->Td = b->Td; cx->err = cudaSuccess; cx->where = "";
+  cx->B = b->B; cx->Te = Te; cx->Td = b->Td; cx->err = cudaSuccess; cx->where = ""; cx->launches = 0;
   return T5_OK;
 }
 
 int end_call(t5_handle* h, Ctx& cx) {
+  h->launches_last_call = cx.launches;
   if (cx.err != cudaSuccess)
     return fail(h, T5_ERR_CUDA, "%s: %s", cx.where, cudaGetErrorString(cx.err));
   return T5_OK;
@@ -588,6 +634,8 @@ int t5_create(const t5_config* cfg, t5_handle** out) {
 }
 
 int t5_destroy(t5_handle* h) {
+  if (h)
+    for (cudaEvent_t e : h->prof_events) cudaEventDestroy(e);
   delete h;
   return T5_OK;
 }
@@ -656,10 +704,10 @@ int t5_train_step_fwd_bwd(t5_handle* h, const void* d_params, const t5_batch* ba
   if (c.arch == 0) encoder_forward(cx, batch);
   decoder_forward(cx, c.arch == 0 ? w.enc_out : nullptr, w.logits);
   CK(cudaMemsetAsync(w.sums, 0, 16, cx.st), "memset sums");
-  CK(launch_xent(c.dtype, w.logits, batch->d_dec_targets, cx.B * cx.Td, c.vocab, c.z_loss, w.W_f, w.sums, w.lse_tok,
+  CKL(CAT_XENT, 1, launch_xent(c.dtype, w.logits, batch->d_dec_targets, cx.B * cx.Td, c.vocab, c.z_loss, w.W_f, w.sums, w.lse_tok,
                  cx.st),
      "xent");
-  CK(launch_finalize_loss(w.sums, w.W_f, d_loss4, cx.st), "finalize loss");
+  CKL(CAT_MISC, 1, launch_finalize_loss(w.sums, w.W_f, d_loss4, cx.st), "finalize loss");
   backward(cx, batch);
   return end_call(h, cx);
 }
@@ -701,6 +749,35 @@ int t5_device_status(t5_handle* h, const void* d_workspace, void* stream) {
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) return fail(h, T5_ERR_CUDA, "device_status: %s", cudaGetErrorString(e));
   if (status != 0) return fail(h, T5_ERR_DEVICE_TIMEOUT, "a bounded device-side wait ran out (code %d)", status);
+  return T5_OK;
+}
+
+int t5_profile_enable(t5_handle* h, int32_t on) {
+  if (!h) return T5_ERR_NULL;
+  h->prof_on = on != 0;
+  h->prof_cat.clear();
+  for (int i = 0; i < 8; ++i) { h->prof_flops[i] = 0; h->prof_launches[i] = 0; }
+  return T5_OK;
+}
+
+int t5_profile_read(t5_handle* h, double ms[8], double flops[8], int64_t launches[8]) {
+  if (!h || !ms || !flops || !launches) return T5_ERR_NULL;
+  for (int i = 0; i < 8; ++i) { ms[i] = 0; flops[i] = h->prof_flops[i]; launches[i] = h->prof_launches[i]; }
+  for (size_t i = 0; i < h->prof_cat.size(); ++i) {
+    cudaError_t e = cudaEventSynchronize(h->prof_events[2 * i + 1]);
+    float t = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&t, h->prof_events[2 * i], h->prof_events[2 * i + 1]);
+    if (e != cudaSuccess) return fail(h, T5_ERR_CUDA, "profile_read: %s", cudaGetErrorString(e));
+    ms[h->prof_cat[i]] += t;
+  }
+  h->prof_cat.clear();
+  for (int i = 0; i < 8; ++i) { h->prof_flops[i] = 0; h->prof_launches[i] = 0; }
+  return T5_OK;
+}
+
+int t5_launch_count(const t5_handle* h, int64_t* n) {
+  if (!h || !n) return T5_ERR_NULL;
+  *n = h->launches_last_call;
   return T5_OK;
 }
 
