@@ -187,6 +187,23 @@ T5_API int t5_gemm(int32_t dtype, int32_t impl, int32_t M, int32_t N, int32_t K,
             int32_t b_kmajor, void* d_D, int32_t ldd, int32_t out_f32, int32_t accumulate,
             void* stream);
 
+/* One attention call on raw buffers (forward, or backward given the forward's
+ * outputs):  S_ij = scale q_i.k_j + bias_delta[h, j - i + Tq - 1], masked by
+ * the position codes (and j <= i when causal), P = softmax_j, O = P V,
+ * lse = log sum_j exp S.  Rows of q/o/do/dq are (b*Tq + i), rows of k/v/dk/dv
+ * are (b*Tk + j); head h occupies columns [h*d_kv, (h+1)*d_kv); ld* are row
+ * strides in elements.  d_bias_delta [H, Tq+Tk-1] may be NULL.  Backward writes
+ * dq, dk, dv, uses d_delta [B,H,Tq] as scratch and ADDS dS summed along
+ * diagonals into d_dbias_delta (may be NULL).  impl 0 = SIMT kernels,
+ * 1 = tcgen05 kernels (bfloat16, d_kv 64 or 128). */
+T5_API int t5_attention(int32_t dtype, int32_t impl, int32_t backward, int32_t B, int32_t H, int32_t Tq,
+                        int32_t Tk, int32_t d_kv, int32_t causal, float scale, const void* d_q, int32_t ldq,
+                        const void* d_k, int32_t ldk, const void* d_v, int32_t ldv, void* d_o, int32_t ldo,
+                        float* d_lse, const int32_t* d_code_q, const int32_t* d_code_k,
+                        const float* d_bias_delta, const void* d_do, int32_t lddo, void* d_dq, int32_t lddq,
+                        void* d_dk, int32_t lddk, void* d_dv, int32_t lddv, float* d_delta,
+                        float* d_dbias_delta, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

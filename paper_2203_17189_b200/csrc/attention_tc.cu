@@ -1,0 +1,829 @@
+// Attention on the tcgen05 tensor cores (bf16 operands, float32 accumulation in
+// tensor memory), forward and backward, with the relative-position bias and the
+// padding / segment / causal masks applied inside the softmax.
+//
+//   S_ij = scale q_i.k_j + bias_delta[h, j-i];  P = softmax_j over valid keys;  O = P V.
+//   backward (P recomputed from the saved log-sum-exp):
+//     dP = dO V^T,  dS = P (dP - delta_i),  dQ = scale dS K,  dK = scale dS^T Q,  dV = P^T dO,
+//     dbias_delta[h, j-i] += dS_ij.
+//
+// All three kernels use 128 threads (thread r owns tensor-memory lane r = one row of
+// the score tile), TMA loads into 128-byte-swizzled tiles, one elected thread issuing
+// the MMAs, and bounded mbarrier waits.  Several CTAs share an SM so that one CTA's
+// softmax overlaps another CTA's MMAs.
+//   forward : CTA = 128 queries x all keys (128-key tiles); online max/sum, output rows
+//             rescaled in registers.
+//   dQ      : CTA = 128 queries x all keys (64-key tiles); dQ accumulates in tensor memory;
+//             dS is also reduced along diagonals into the bias gradient.
+//   dK, dV  : CTA = 128 keys x all queries (64-query tiles), scores transposed (thread = key);
+//             dK and dV accumulate in tensor memory.
+#include "common.cuh"
+#include "tc_common.cuh"
+
+#include <math.h>
+
+namespace {
+
+using namespace tc;
+
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct TcParams {
+  const void* O;        // forward: output (written); backward: unused
+  void* out0;           // forward: O; dQ kernel: dQ; dKV kernel: dK
+  void* out1;           // dKV kernel: dV
+  int ld0, ld1;
+  float* lse;           // [B,H,Tq] written by forward, read by backward
+  const float* delta;   // [B,H,Tq]
+  const int* code_q;
+  const int* code_k;
+  const float* bias_delta;   // [H, Tq+Tk-1] or NULL
+  float* dbias_delta;        // [H, Tq+Tk-1] or NULL
+  int B, H, Tq, Tk, causal;
+  float scale;
+  int* status;
+};
+
+__device__ __forceinline__ uint64_t desc_k(uint32_t addr) { return make_desc(addr, 16, 1024); }
+__device__ __forceinline__ uint64_t desc_mn(uint32_t addr, uint32_t lbo) { return make_desc(addr, lbo, 1024); }
+
+// Writes 8 consecutive bf16 of row `row` (columns [col8*8, col8*8+8) of a 64-column chunk) into a
+// 128-byte-swizzled K-major tile: 16-byte piece index is XORed with (row % 8).
+__device__ __forceinline__ void store_swizzled_16B(unsigned char* tile, int row, int piece, uint4 v) {
+  *reinterpret_cast<uint4*>(tile + row * 128 + ((piece ^ (row & 7)) << 4)) = v;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&t);
+}
+
+struct Bars {
+  uint64_t ld[4];      // TMA barriers (meaning per kernel)
+  uint64_t mma[2];     // MMA completion barriers
+  uint32_t tmem;
+  int abort_flag;
+};
+
+// ============================================================================ forward
+template <int DK>
+struct FwdLayout {
+  static constexpr int kTile = 128 * DK * 2;          // Q, K or V tile bytes
+  static constexpr int kP = 128 * 128 * 2;
+  static constexpr int kQ = 0, kK = kTile, kV = 2 * kTile, kPo = 3 * kTile, kMisc = 3 * kTile + kP;
+  static int bytes(int Tk) {
+    int tkp = (Tk + 127) / 128 * 128;
+    return kMisc + (tkp + 128) * 4 + tkp * 4 + (int)sizeof(Bars) + 1024 + 64;
+  }
+};
+
+template <int DK>
+__global__ void __launch_bounds__(128)
+attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
+                   const __grid_constant__ CUtensorMap mv, TcParams p) {
+  using L = FwdLayout<DK>;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const int tkp = (p.Tk + 127) / 128 * 128;
+  float* bias_s = (float*)(smem + L::kMisc);          // [tkp + 128]
+  int* codes_s = (int*)(bias_s + tkp + 128);          // [tkp]
+  Bars* bars = (Bars*)(((uintptr_t)(codes_s + tkp) + 15) & ~(uintptr_t)15);
+  volatile int* abort_flag = &bars->abort_flag;
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * 128;
+  int n_kt = (p.Tk + 127) / 128;
+  if (p.causal) n_kt = min(n_kt, (q0 + 127) / 128 + 1);
+  constexpr uint32_t kTmemCols = 256;
+
+  if (tid == 0) {
+    for (int i = 0; i < 4; ++i) mbar_init(&bars->ld[i], 1);
+    for (int i = 0; i < 2; ++i) mbar_init(&bars->mma[i], 1);
+    bars->abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 0) tmem_alloc(&bars->tmem, kTmemCols);
+  const int span = p.Tq + p.Tk - 1;
+  for (int w = tid; w < tkp + 128; w += 128) {
+    int g = w - 127 - q0 + p.Tq - 1;
+    bias_s[w] = (p.bias_delta && g >= 0 && g < span) ? p.bias_delta[(int64_t)h * span + g] * kLog2e : 0.f;
+  }
+  for (int j = tid; j < tkp; j += 128) codes_s[j] = j < p.Tk ? p.code_k[b * p.Tk + j] : 0;
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem;
+  const uint32_t sQ = smem_u32(smem + L::kQ), sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV),
+                 sP = smem_u32(smem + L::kPo);
+  uint64_t* bar_k = &bars->ld[0];
+  uint64_t* bar_v = &bars->ld[1];
+  uint64_t* bar_m = &bars->mma[0];
+
+  if (tid == 0) {
+    mbar_arrive_expect_tx(bar_k, 2 * L::kTile);
+#pragma unroll
+    for (int c = 0; c < DK / 64; ++c) {
+      tma_load_3d(smem + L::kQ + c * 16384, &mq, h * DK + c * 64, q0, b, bar_k);
+      tma_load_3d(smem + L::kK + c * 16384, &mk, h * DK + c * 64, 0, b, bar_k);
+    }
+    mbar_arrive_expect_tx(bar_v, L::kTile);
+#pragma unroll
+    for (int c = 0; c < DK / 64; ++c) tma_load_3d(smem + L::kV + c * 16384, &mv, h * DK + c * 64, 0, b, bar_v);
+  }
+
+  const int i = q0 + tid;
+  const int cq = i < p.Tq ? p.code_q[b * p.Tq + i] : 0;
+  float m_run = -INFINITY, l_run = 0.f;
+  float o[DK];
+#pragma unroll
+  for (int d = 0; d < DK; ++d) o[d] = 0.f;
+  const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+  const float sc2 = p.scale * kLog2e;
+  uint32_t ph_k = 0, ph_v = 0, ph_m = 0;
+  bool ok = true, pend_k = true, pend_v = true;      // pend_*: a load of that tile is in flight (thread 0 only)
+  constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
+  constexpr uint32_t idesc_pv = make_idesc(128, DK, false, true);
+
+  for (int t = 0; t < n_kt && ok; ++t) {
+    const int k0 = t * 128;
+    if (tid == 0) {
+      if (mbar_wait(bar_k, ph_k, abort_flag, p.status, 11)) {
+        ph_k ^= 1;
+        pend_k = false;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < DK / 16; ++kk) {
+          uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
+          umma_bf16(tmem_base, desc_k(sQ + off), desc_k(sK + off), idesc_s, kk != 0);
+        }
+        umma_commit(bar_m);
+      }
+    }
+    ok = mbar_wait(bar_m, ph_m, abort_flag, p.status, 12);
+    ph_m ^= 1;
+    if (!ok) break;
+    tc_fence_after();
+    if (tid == 0 && t + 1 < n_kt) {     // K tile is free again: fetch the next one
+      pend_k = true;
+      mbar_arrive_expect_tx(bar_k, L::kTile);
+#pragma unroll
+      for (int c = 0; c < DK / 64; ++c)
+        tma_load_3d(smem + L::kK + c * 16384, &mk, h * DK + c * 64, k0 + 128, b, bar_k);
+    }
+    // pass 1: row maximum of the masked, biased scores (in log2 units)
+    float mt = -INFINITY;
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+      uint32_t r[32];
+      tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, r);
+      tmem_wait_ld();
+#pragma unroll
+      for (int jj = 0; jj < 32; ++jj) {
+        int j = k0 + c * 32 + jj;
+        int ck = codes_s[j];
+        bool valid = ck != 0 && ck == cq && (!p.causal || j <= i);
+        float s = __uint_as_float(r[jj]) * sc2 + bias_s[j - tid + 127];
+        mt = valid ? fmaxf(mt, s) : mt;
+      }
+    }
+    const float m_new = fmaxf(m_run, mt);
+    const float corr = m_run == -INFINITY ? 0.f : exp2f(m_run - m_new);
+    float lsum = 0.f;
+    // pass 2: probabilities (bf16) into the swizzled P tile
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+      uint32_t r[32];
+      tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, r);
+      tmem_wait_ld();
+      float pv[32];
+#pragma unroll
+      for (int jj = 0; jj < 32; ++jj) {
+        int j = k0 + c * 32 + jj;
+        int ck = codes_s[j];
+        bool valid = ck != 0 && ck == cq && (!p.causal || j <= i);
+        float s = __uint_as_float(r[jj]) * sc2 + bias_s[j - tid + 127];
+        float e = valid ? exp2f(s - m_new) : 0.f;
+        pv[jj] = e;
+        lsum += e;
+      }
+      unsigned char* chunk = smem + L::kPo + (c >> 1) * 16384;
+#pragma unroll
+      for (int q8 = 0; q8 < 4; ++q8) {
+        uint4 v;
+        v.x = pack_bf16(pv[q8 * 8 + 0], pv[q8 * 8 + 1]);
+        v.y = pack_bf16(pv[q8 * 8 + 2], pv[q8 * 8 + 3]);
+        v.z = pack_bf16(pv[q8 * 8 + 4], pv[q8 * 8 + 5]);
+        v.w = pack_bf16(pv[q8 * 8 + 6], pv[q8 * 8 + 7]);
+        store_swizzled_16B(chunk, tid, (c & 1) * 4 + q8, v);
+      }
+    }
+    l_run = l_run * corr + lsum;
+    m_run = m_new;
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      if (mbar_wait(bar_v, ph_v, abort_flag, p.status, 13)) {
+        ph_v ^= 1;
+        pend_v = false;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          umma_bf16(tmem_base + 128, desc_k(sP + (ks >> 2) * 16384 + (ks & 3) * 32), desc_mn(sV + ks * 2048, 16384),
+                    idesc_pv, ks != 0);
+        umma_commit(bar_m);
+      }
+    }
+    ok = mbar_wait(bar_m, ph_m, abort_flag, p.status, 14);
+    ph_m ^= 1;
+    if (!ok) break;
+    tc_fence_after();
+    if (tid == 0 && t + 1 < n_kt) {
+      pend_v = true;
+      mbar_arrive_expect_tx(bar_v, L::kTile);
+#pragma unroll
+      for (int c = 0; c < DK / 64; ++c)
+        tma_load_3d(smem + L::kV + c * 16384, &mv, h * DK + c * 64, k0 + 128, b, bar_v);
+    }
+#pragma unroll
+    for (int c = 0; c < DK / 32; ++c) {
+      uint32_t r[32];
+      tmem_ld_32x32b_x32(tmem_base + lane_off + 128 + c * 32, r);
+      tmem_wait_ld();
+#pragma unroll
+      for (int jj = 0; jj < 32; ++jj) o[c * 32 + jj] = o[c * 32 + jj] * corr + __uint_as_float(r[jj]);
+    }
+    tc_fence_before();
+  }
+
+  if (ok && i < p.Tq) {
+    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+    bf16* orow = (bf16*)p.out0 + (int64_t)(b * p.Tq + i) * p.ld0 + h * DK;
+#pragma unroll
+    for (int d = 0; d < DK; d += 8) {
+      uint4 v;
+      v.x = pack_bf16(o[d] * inv, o[d + 1] * inv);
+      v.y = pack_bf16(o[d + 2] * inv, o[d + 3] * inv);
+      v.z = pack_bf16(o[d + 4] * inv, o[d + 5] * inv);
+      v.w = pack_bf16(o[d + 6] * inv, o[d + 7] * inv);
+      *reinterpret_cast<uint4*>(orow + d) = v;
+    }
+    // natural-log log-sum-exp of the (unscaled-by-log2e) scores
+    p.lse[(int64_t)(b * p.H + h) * p.Tq + i] = l_run > 0.f ? (m_run + log2f(l_run)) / kLog2e : -INFINITY;
+  }
+  if (!ok && tid == 0) {   // let TMA loads that are still in flight land before the CTA exits
+    long long t0 = clock64();
+    while (pend_k && !mbar_try_wait(bar_k, ph_k) && clock64() - t0 < kWaitCycles) {}
+    while (pend_v && !mbar_try_wait(bar_v, ph_v) && clock64() - t0 < kWaitCycles) {}
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ============================================================================ backward: dQ (+ dbias)
+template <int DK>
+struct DqLayout {
+  static constexpr int kQ = 0, kDO = 128 * DK * 2, kKV0 = 2 * 128 * DK * 2;
+  static constexpr int kKVTile = 64 * DK * 2;                   // one K or V tile (64 keys)
+  static constexpr int kStage = 2 * kKVTile;                    // K then V
+  static constexpr int kDS = kKV0 + 2 * kStage;                 // [128 x 64] bf16
+  static constexpr int kMisc = kDS + 128 * 64 * 2;
+  static int bytes(int Tk) {
+    int tkp = (Tk + 63) / 64 * 64;
+    return kMisc + 2 * (tkp + 128) * 4 + tkp * 4 + (int)sizeof(Bars) + 1024 + 64;
+  }
+};
+
+template <int DK>
+__global__ void __launch_bounds__(128)
+attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mdo,
+                      const __grid_constant__ CUtensorMap mk, const __grid_constant__ CUtensorMap mv, TcParams p) {
+  using L = DqLayout<DK>;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const int tkp = (p.Tk + 63) / 64 * 64;
+  float* bias_s = (float*)(smem + L::kMisc);          // [tkp + 128]
+  float* dbias_s = bias_s + tkp + 128;                // [tkp + 128]
+  int* codes_s = (int*)(dbias_s + tkp + 128);         // [tkp]
+  Bars* bars = (Bars*)(((uintptr_t)(codes_s + tkp) + 15) & ~(uintptr_t)15);
+  volatile int* abort_flag = &bars->abort_flag;
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * 128;
+  int n_kt = (p.Tk + 63) / 64;
+  if (p.causal) n_kt = min(n_kt, (q0 + 127) / 64 + 1);
+  constexpr uint32_t kTmemCols = 256;
+  const bool want_db = p.dbias_delta != nullptr;
+
+  if (tid == 0) {
+    for (int i = 0; i < 4; ++i) mbar_init(&bars->ld[i], 1);
+    for (int i = 0; i < 2; ++i) mbar_init(&bars->mma[i], 1);
+    bars->abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 0) tmem_alloc(&bars->tmem, kTmemCols);
+  const int span = p.Tq + p.Tk - 1;
+  for (int w = tid; w < tkp + 128; w += 128) {
+    int g = w - 127 - q0 + p.Tq - 1;
+    bias_s[w] = (p.bias_delta && g >= 0 && g < span) ? p.bias_delta[(int64_t)h * span + g] * kLog2e : 0.f;
+    dbias_s[w] = 0.f;
+  }
+  for (int j = tid; j < tkp; j += 128) codes_s[j] = j < p.Tk ? p.code_k[b * p.Tk + j] : 0;
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem;
+  const uint32_t sQ = smem_u32(smem + L::kQ), sDO = smem_u32(smem + L::kDO), sDS = smem_u32(smem + L::kDS);
+  uint64_t* bar_q = &bars->ld[0];        // Q and dO
+  uint64_t* bar_kv = &bars->ld[1];       // [2] stages: ld[1], ld[2]
+  uint64_t* bar_m = &bars->mma[0];       // S and dP ready
+  uint64_t* bar_dq = &bars->mma[1];      // dQ MMA of the tile done
+
+  auto load_kv = [&](int t) {
+    int st = t & 1;
+    unsigned char* base = smem + L::kKV0 + st * L::kStage;
+    mbar_arrive_expect_tx(&bar_kv[st], L::kStage);
+#pragma unroll
+    for (int c = 0; c < DK / 64; ++c) {
+      tma_load_3d(base + c * 8192, &mk, h * DK + c * 64, t * 64, b, &bar_kv[st]);
+      tma_load_3d(base + L::kKVTile + c * 8192, &mv, h * DK + c * 64, t * 64, b, &bar_kv[st]);
+    }
+  };
+  if (tid == 0) {
+    mbar_arrive_expect_tx(bar_q, 2 * 128 * DK * 2);
+#pragma unroll
+    for (int c = 0; c < DK / 64; ++c) {
+      tma_load_3d(smem + L::kQ + c * 16384, &mq, h * DK + c * 64, q0, b, bar_q);
+      tma_load_3d(smem + L::kDO + c * 16384, &mdo, h * DK + c * 64, q0, b, bar_q);
+    }
+    load_kv(0);
+  }
+
+  const int i = q0 + tid;
+  const bool row_in = i < p.Tq;
+  const int cq = row_in ? p.code_q[b * p.Tq + i] : 0;
+  const float lse2 = row_in ? p.lse[(int64_t)(b * p.H + h) * p.Tq + i] * kLog2e : -INFINITY;
+  const float dl = row_in ? p.delta[(int64_t)(b * p.H + h) * p.Tq + i] : 0.f;
+  const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+  const float sc2 = p.scale * kLog2e;
+  uint32_t ph_kv[2] = {0, 0}, ph_m = 0, ph_dq = 0;
+  bool ok = true;
+  constexpr uint32_t idesc_s = make_idesc(128, 64, false, false);
+  constexpr uint32_t idesc_dq = make_idesc(128, DK, false, true);
+
+  if (tid == 0) ok = mbar_wait(bar_q, 0, abort_flag, p.status, 21);
+
+  for (int t = 0; t < n_kt && ok; ++t) {
+    const int k0 = t * 64, st = t & 1;
+    const uint32_t sK = smem_u32(smem + L::kKV0 + st * L::kStage), sV = sK + L::kKVTile;
+    if (tid == 0) {
+      if (t + 1 < n_kt) load_kv(t + 1);      // the other stage was released by the dQ wait of tile t-1
+      if (mbar_wait(&bar_kv[st], ph_kv[st], abort_flag, p.status, 22)) {
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < DK / 16; ++kk) {
+          uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
+          umma_bf16(tmem_base, desc_k(sQ + oa), desc_k(sK + ob), idesc_s, kk != 0);
+        }
+#pragma unroll
+        for (int kk = 0; kk < DK / 16; ++kk) {
+          uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
+          umma_bf16(tmem_base + 64, desc_k(sDO + oa), desc_k(sV + ob), idesc_s, kk != 0);
+        }
+        umma_commit(bar_m);
+      }
+    }
+    ph_kv[st] ^= 1;
+    ok = mbar_wait(bar_m, ph_m, abort_flag, p.status, 23);
+    ph_m ^= 1;
+    if (!ok) break;
+    tc_fence_after();
+#pragma unroll 1
+    for (int c = 0; c < 2; ++c) {
+      uint32_t rs[32], rp[32];
+      tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, rs);
+      tmem_ld_32x32b_x32(tmem_base + lane_off + 64 + c * 32, rp);
+      tmem_wait_ld();
+      float ds[32];
+#pragma unroll
+      for (int jj = 0; jj < 32; ++jj) {
+        int j = k0 + c * 32 + jj;
+        int ck = codes_s[j];
+        bool valid = ck != 0 && ck == cq && (!p.causal || j <= i) && lse2 != -INFINITY;
+        float s = __uint_as_float(rs[jj]) * sc2 + bias_s[j - tid + 127];
+        float pr = valid ? exp2f(s - lse2) : 0.f;
+        float v = pr * (__uint_as_float(rp[jj]) - dl);
+        ds[jj] = v;
+        if (want_db && valid) atomicAdd(&dbias_s[j - tid + 127], v);
+      }
+#pragma unroll
+      for (int q8 = 0; q8 < 4; ++q8) {
+        uint4 v;
+        v.x = pack_bf16(ds[q8 * 8 + 0], ds[q8 * 8 + 1]);
+        v.y = pack_bf16(ds[q8 * 8 + 2], ds[q8 * 8 + 3]);
+        v.z = pack_bf16(ds[q8 * 8 + 4], ds[q8 * 8 + 5]);
+        v.w = pack_bf16(ds[q8 * 8 + 6], ds[q8 * 8 + 7]);
+        store_swizzled_16B(smem + L::kDS, tid, c * 4 + q8, v);
+      }
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks)
+        umma_bf16(tmem_base + 128, desc_k(sDS + ks * 32), desc_mn(sK + ks * 2048, 8192), idesc_dq, (t | ks) != 0);
+      umma_commit(bar_dq);
+    }
+    ok = mbar_wait(bar_dq, ph_dq, abort_flag, p.status, 24);   // dS tile and this K/V stage are free again
+    ph_dq ^= 1;
+  }
+
+  if (ok) {
+    tc_fence_after();
+    bf16* drow = (bf16*)p.out0 + (int64_t)(b * p.Tq + i) * p.ld0 + h * DK;
+#pragma unroll
+    for (int c = 0; c < DK / 32; ++c) {
+      uint32_t r[32];
+      tmem_ld_32x32b_x32(tmem_base + lane_off + 128 + c * 32, r);
+      tmem_wait_ld();
+      if (row_in) {
+#pragma unroll
+        for (int d = 0; d < 32; d += 8) {
+          uint4 v;
+          v.x = pack_bf16(p.scale * __uint_as_float(r[d]), p.scale * __uint_as_float(r[d + 1]));
+          v.y = pack_bf16(p.scale * __uint_as_float(r[d + 2]), p.scale * __uint_as_float(r[d + 3]));
+          v.z = pack_bf16(p.scale * __uint_as_float(r[d + 4]), p.scale * __uint_as_float(r[d + 5]));
+          v.w = pack_bf16(p.scale * __uint_as_float(r[d + 6]), p.scale * __uint_as_float(r[d + 7]));
+          *reinterpret_cast<uint4*>(drow + c * 32 + d) = v;
+        }
+      }
+    }
+  }
+  if (!ok && tid == 0) {   // a wait ran out: give loads still in flight a bounded time to land
+    long long t0 = clock64();
+    while (clock64() - t0 < 4000000ll) {}
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (ok && want_db) {
+    for (int w = tid; w < tkp + 128; w += 128) {
+      float v = dbias_s[w];
+      int g = w - 127 - q0 + p.Tq - 1;
+      if (v != 0.f && g >= 0 && g < span) atomicAdd(&p.dbias_delta[(int64_t)h * span + g], v);
+    }
+  }
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ============================================================================ backward: dK, dV
+template <int DK>
+struct DkvLayout {
+  static constexpr int kK = 0, kV = 128 * DK * 2, kQD0 = 2 * 128 * DK * 2;
+  static constexpr int kQTile = 64 * DK * 2;                    // one Q or dO tile (64 queries)
+  static constexpr int kStage = 2 * kQTile;                     // Q then dO
+  static constexpr int kPt = kQD0 + 2 * kStage;                 // [128 keys x 64 queries] bf16
+  static constexpr int kDSt = kPt + 128 * 64 * 2;
+  static constexpr int kMisc = kDSt + 128 * 64 * 2;
+  static int bytes(int Tq) {
+    int tqp = (Tq + 63) / 64 * 64;
+    return kMisc + (tqp + 128) * 4 + 3 * tqp * 4 + (int)sizeof(Bars) + 1024 + 64;
+  }
+};
+
+template <int DK>
+__global__ void __launch_bounds__(128)
+attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mdo,
+                       const __grid_constant__ CUtensorMap mk, const __grid_constant__ CUtensorMap mv, TcParams p) {
+  using L = DkvLayout<DK>;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const int tqp = (p.Tq + 63) / 64 * 64;
+  float* bias_s = (float*)(smem + L::kMisc);          // [tqp + 128], indexed by (tid - i_local + tqp... see below)
+  float* lse_s = bias_s + tqp + 128;                  // [tqp]  (log2 units)
+  float* dl_s = lse_s + tqp;                          // [tqp]
+  int* codes_s = (int*)(dl_s + tqp);                  // [tqp] query codes
+  Bars* bars = (Bars*)(((uintptr_t)(codes_s + tqp) + 15) & ~(uintptr_t)15);
+  volatile int* abort_flag = &bars->abort_flag;
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int b = blockIdx.z, h = blockIdx.y, k0 = blockIdx.x * 128;
+  const int n_qt = (p.Tq + 63) / 64;
+  const int t_begin = p.causal ? k0 / 64 : 0;          // queries before k0 see none of these keys
+  constexpr uint32_t kTmemCols = DK == 64 ? 256 : 512;
+
+  if (tid == 0) {
+    for (int i = 0; i < 4; ++i) mbar_init(&bars->ld[i], 1);
+    for (int i = 0; i < 2; ++i) mbar_init(&bars->mma[i], 1);
+    bars->abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 0) tmem_alloc(&bars->tmem, kTmemCols);
+  const int span = p.Tq + p.Tk - 1;
+  // distance of (key j = k0 + tid, query i): j - i ; window index w = tid - i + tqp  in [1, tqp + 127]
+  for (int w = tid; w < tqp + 128; w += 128) {
+    int g = (w - tqp) + k0 + p.Tq - 1;
+    bias_s[w] = (p.bias_delta && g >= 0 && g < span) ? p.bias_delta[(int64_t)h * span + g] * kLog2e : 0.f;
+  }
+  for (int q = tid; q < tqp; q += 128) {
+    bool in = q < p.Tq;
+    lse_s[q] = in ? p.lse[(int64_t)(b * p.H + h) * p.Tq + q] * kLog2e : -INFINITY;
+    dl_s[q] = in ? p.delta[(int64_t)(b * p.H + h) * p.Tq + q] : 0.f;
+    codes_s[q] = in ? p.code_q[b * p.Tq + q] : 0;
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem;
+  const uint32_t sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV), sPt = smem_u32(smem + L::kPt),
+                 sDSt = smem_u32(smem + L::kDSt);
+  uint64_t* bar_kv = &bars->ld[0];
+  uint64_t* bar_qd = &bars->ld[1];       // [2] stages
+  uint64_t* bar_m = &bars->mma[0];
+  uint64_t* bar_acc = &bars->mma[1];
+
+  auto load_qd = [&](int t) {
+    int st = t & 1;
+    unsigned char* base = smem + L::kQD0 + st * L::kStage;
+    mbar_arrive_expect_tx(&bar_qd[st], L::kStage);
+#pragma unroll
+    for (int c = 0; c < DK / 64; ++c) {
+      tma_load_3d(base + c * 8192, &mq, h * DK + c * 64, t * 64, b, &bar_qd[st]);
+      tma_load_3d(base + L::kQTile + c * 8192, &mdo, h * DK + c * 64, t * 64, b, &bar_qd[st]);
+    }
+  };
+  if (tid == 0 && t_begin < n_qt) {
+    mbar_arrive_expect_tx(bar_kv, 2 * 128 * DK * 2);
+#pragma unroll
+    for (int c = 0; c < DK / 64; ++c) {
+      tma_load_3d(smem + L::kK + c * 16384, &mk, h * DK + c * 64, k0, b, bar_kv);
+      tma_load_3d(smem + L::kV + c * 16384, &mv, h * DK + c * 64, k0, b, bar_kv);
+    }
+    load_qd(t_begin);
+  }
+
+  const int j = k0 + tid;
+  const bool row_in = j < p.Tk;
+  const int ck = row_in ? p.code_k[b * p.Tk + j] : 0;
+  const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+  const float sc2 = p.scale * kLog2e;
+  uint32_t ph_qd[2] = {0, 0}, ph_m = 0, ph_acc = 0;
+  bool ok = true;
+  constexpr uint32_t idesc_s = make_idesc(128, 64, false, false);
+  constexpr uint32_t idesc_acc = make_idesc(128, DK, false, true);
+  if (tid == 0 && t_begin < n_qt) ok = mbar_wait(bar_kv, 0, abort_flag, p.status, 31);
+
+  for (int t = t_begin; t < n_qt && ok; ++t) {
+    const int qb = t * 64;
+    const uint32_t sQ = smem_u32(smem + L::kQD0 + (t & 1) * L::kStage), sDO = sQ + L::kQTile;
+    if (tid == 0) {
+      if (t + 1 < n_qt) load_qd(t + 1);
+      if (mbar_wait(&bar_qd[t & 1], ph_qd[t & 1], abort_flag, p.status, 32)) {
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < DK / 16; ++kk) {
+          uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
+          umma_bf16(tmem_base, desc_k(sK + oa), desc_k(sQ + ob), idesc_s, kk != 0);
+        }
+#pragma unroll
+        for (int kk = 0; kk < DK / 16; ++kk) {
+          uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
+          umma_bf16(tmem_base + 64, desc_k(sV + oa), desc_k(sDO + ob), idesc_s, kk != 0);
+        }
+        umma_commit(bar_m);
+      }
+    }
+    ph_qd[t & 1] ^= 1;
+    ok = mbar_wait(bar_m, ph_m, abort_flag, p.status, 33);
+    ph_m ^= 1;
+    if (!ok) break;
+    tc_fence_after();
+#pragma unroll 1
+    for (int c = 0; c < 2; ++c) {
+      uint32_t rs[32], rp[32];
+      tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, rs);
+      tmem_ld_32x32b_x32(tmem_base + lane_off + 64 + c * 32, rp);
+      tmem_wait_ld();
+      float pt[32], ds[32];
+#pragma unroll
+      for (int ii = 0; ii < 32; ++ii) {
+        int q = qb + c * 32 + ii;
+        int cq = codes_s[q];
+        float lse2 = lse_s[q];
+        bool valid = ck != 0 && ck == cq && (!p.causal || j <= q) && lse2 != -INFINITY;
+        float s = __uint_as_float(rs[ii]) * sc2 + bias_s[tid - q + tqp];
+        float pr = valid ? exp2f(s - lse2) : 0.f;
+        pt[ii] = pr;
+        ds[ii] = pr * (__uint_as_float(rp[ii]) - dl_s[q]);
+      }
+#pragma unroll
+      for (int q8 = 0; q8 < 4; ++q8) {
+        uint4 v;
+        v.x = pack_bf16(pt[q8 * 8 + 0], pt[q8 * 8 + 1]);
+        v.y = pack_bf16(pt[q8 * 8 + 2], pt[q8 * 8 + 3]);
+        v.z = pack_bf16(pt[q8 * 8 + 4], pt[q8 * 8 + 5]);
+        v.w = pack_bf16(pt[q8 * 8 + 6], pt[q8 * 8 + 7]);
+        store_swizzled_16B(smem + L::kPt, tid, c * 4 + q8, v);
+        v.x = pack_bf16(ds[q8 * 8 + 0], ds[q8 * 8 + 1]);
+        v.y = pack_bf16(ds[q8 * 8 + 2], ds[q8 * 8 + 3]);
+        v.z = pack_bf16(ds[q8 * 8 + 4], ds[q8 * 8 + 5]);
+        v.w = pack_bf16(ds[q8 * 8 + 6], ds[q8 * 8 + 7]);
+        store_swizzled_16B(smem + L::kDSt, tid, c * 4 + q8, v);
+      }
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+      const uint32_t first = (t == t_begin) ? 0u : 1u;
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks)
+        umma_bf16(tmem_base + 128, desc_k(sPt + ks * 32), desc_mn(sDO + ks * 2048, 8192), idesc_acc, first | ks);
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks)
+        umma_bf16(tmem_base + 128 + DK, desc_k(sDSt + ks * 32), desc_mn(sQ + ks * 2048, 8192), idesc_acc,
+                  first | ks);
+      umma_commit(bar_acc);
+    }
+    ok = mbar_wait(bar_acc, ph_acc, abort_flag, p.status, 34);
+    ph_acc ^= 1;
+  }
+
+  if (ok) {
+    tc_fence_after();
+    bf16* krow = (bf16*)p.out0 + (int64_t)(b * p.Tk + j) * p.ld0 + h * DK;
+    bf16* vrow = (bf16*)p.out1 + (int64_t)(b * p.Tk + j) * p.ld1 + h * DK;
+    const bool any = t_begin < n_qt;
+#pragma unroll
+    for (int c = 0; c < DK / 32; ++c) {
+      uint32_t rv[32], rk[32];
+      if (any) {
+        tmem_ld_32x32b_x32(tmem_base + lane_off + 128 + c * 32, rv);
+        tmem_ld_32x32b_x32(tmem_base + lane_off + 128 + DK + c * 32, rk);
+        tmem_wait_ld();
+      } else {
+#pragma unroll
+        for (int d = 0; d < 32; ++d) rv[d] = rk[d] = 0u;
+      }
+      if (row_in) {
+#pragma unroll
+        for (int d = 0; d < 32; d += 8) {
+          uint4 v;
+          v.x = pack_bf16(__uint_as_float(rv[d]), __uint_as_float(rv[d + 1]));
+          v.y = pack_bf16(__uint_as_float(rv[d + 2]), __uint_as_float(rv[d + 3]));
+          v.z = pack_bf16(__uint_as_float(rv[d + 4]), __uint_as_float(rv[d + 5]));
+          v.w = pack_bf16(__uint_as_float(rv[d + 6]), __uint_as_float(rv[d + 7]));
+          *reinterpret_cast<uint4*>(vrow + c * 32 + d) = v;
+          v.x = pack_bf16(p.scale * __uint_as_float(rk[d]), p.scale * __uint_as_float(rk[d + 1]));
+          v.y = pack_bf16(p.scale * __uint_as_float(rk[d + 2]), p.scale * __uint_as_float(rk[d + 3]));
+          v.z = pack_bf16(p.scale * __uint_as_float(rk[d + 4]), p.scale * __uint_as_float(rk[d + 5]));
+          v.w = pack_bf16(p.scale * __uint_as_float(rk[d + 6]), p.scale * __uint_as_float(rk[d + 7]));
+          *reinterpret_cast<uint4*>(krow + c * 32 + d) = v;
+        }
+      }
+    }
+  }
+  if (!ok && tid == 0) {   // a wait ran out: give loads still in flight a bounded time to land
+    long long t0 = clock64();
+    while (clock64() - t0 < 4000000ll) {}
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ----------------------------------------------------------------------------- delta = rowsum(dO * O)
+template <int DK>
+__global__ void attn_delta_tc_kernel(const bf16* __restrict__ O, int ldo, const bf16* __restrict__ dO, int lddo,
+                                     float* __restrict__ delta, int B, int H, int Tq) {
+  int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (gw >= B * Tq * H) return;
+  int h = gw % H, row = gw / H;
+  int b = row / Tq, i = row % Tq;
+  float s = 0.f;
+#pragma unroll
+  for (int c = 0; c < DK / 64; ++c) {
+    __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(O + (int64_t)row * ldo + h * DK + c * 64 + lane * 2);
+    __nv_bfloat162 g = *reinterpret_cast<const __nv_bfloat162*>(dO + (int64_t)row * lddo + h * DK + c * 64 + lane * 2);
+    float2 fa = __bfloat1622float2(a), fg = __bfloat1622float2(g);
+    s += fa.x * fg.x + fa.y * fg.y;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if (lane == 0) delta[(int64_t)(b * H + h) * Tq + i] = s;
+}
+
+// ----------------------------------------------------------------------------- host side
+// 3-D view [B][T][cols] of a row-major token matrix with row stride ld; box = [1][rows][64 cols]
+bool make_map3(CUtensorMap* m, const void* base, int cols, int T, int B, int ld, int box_rows) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)T, (cuuint64_t)B};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)T * ld * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+TcParams base_params(const AttnArgs& a, int* status) {
+  TcParams p{};
+  p.lse = a.lse; p.delta = a.delta; p.code_q = a.code_q; p.code_k = a.code_k; p.bias_delta = a.bias_delta;
+  p.dbias_delta = a.dbias_delta; p.B = a.B; p.H = a.H; p.Tq = a.Tq; p.Tk = a.Tk; p.causal = a.causal;
+  p.scale = a.scale; p.status = status;
+  return p;
+}
+
+template <int DK>
+cudaError_t fwd_launch(const AttnArgs& a, int* status, cudaStream_t st) {
+  CUtensorMap mq, mk, mv;
+  int I = a.H * DK;
+  if (!make_map3(&mq, a.Q, I, a.Tq, a.B, a.ldq, 128) || !make_map3(&mk, a.K, I, a.Tk, a.B, a.ldk, 128) ||
+      !make_map3(&mv, a.V, I, a.Tk, a.B, a.ldv, 128))
+    return cudaErrorInvalidValue;
+  int smem = FwdLayout<DK>::bytes(a.Tk);
+  cudaError_t e = cudaFuncSetAttribute(attn_fwd_tc_kernel<DK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  TcParams p = base_params(a, status);
+  p.out0 = a.O; p.ld0 = a.ldo;
+  dim3 grid((a.Tq + 127) / 128, a.H, a.B);
+  attn_fwd_tc_kernel<DK><<<grid, 128, smem, st>>>(mq, mk, mv, p);
+  return cudaGetLastError();
+}
+
+template <int DK>
+cudaError_t bwd_launch(const AttnArgs& a, int* status, cudaStream_t st) {
+  int I = a.H * DK;
+  int warps = a.B * a.Tq * a.H;
+  attn_delta_tc_kernel<DK><<<(warps + 7) / 8, 256, 0, st>>>((const bf16*)a.O, a.ldo, (const bf16*)a.dO, a.lddo,
+                                                            a.delta, a.B, a.H, a.Tq);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  TcParams p = base_params(a, status);
+  {
+    CUtensorMap mq, mdo, mk, mv;
+    if (!make_map3(&mq, a.Q, I, a.Tq, a.B, a.ldq, 128) || !make_map3(&mdo, a.dO, I, a.Tq, a.B, a.lddo, 128) ||
+        !make_map3(&mk, a.K, I, a.Tk, a.B, a.ldk, 64) || !make_map3(&mv, a.V, I, a.Tk, a.B, a.ldv, 64))
+      return cudaErrorInvalidValue;
+    int smem = DqLayout<DK>::bytes(a.Tk);
+    e = cudaFuncSetAttribute(attn_bwd_dq_tc_kernel<DK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    p.out0 = a.dQ; p.ld0 = a.lddq;
+    dim3 grid((a.Tq + 127) / 128, a.H, a.B);
+    attn_bwd_dq_tc_kernel<DK><<<grid, 128, smem, st>>>(mq, mdo, mk, mv, p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  {
+    CUtensorMap mq, mdo, mk, mv;
+    if (!make_map3(&mq, a.Q, I, a.Tq, a.B, a.ldq, 64) || !make_map3(&mdo, a.dO, I, a.Tq, a.B, a.lddo, 64) ||
+        !make_map3(&mk, a.K, I, a.Tk, a.B, a.ldk, 128) || !make_map3(&mv, a.V, I, a.Tk, a.B, a.ldv, 128))
+      return cudaErrorInvalidValue;
+    int smem = DkvLayout<DK>::bytes(a.Tq);
+    e = cudaFuncSetAttribute(attn_bwd_dkv_tc_kernel<DK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    p.out0 = a.dK; p.ld0 = a.lddk; p.out1 = a.dV; p.ld1 = a.lddv;
+    dim3 grid((a.Tk + 127) / 128, a.H, a.B);
+    attn_bwd_dkv_tc_kernel<DK><<<grid, 128, smem, st>>>(mq, mdo, mk, mv, p);
+    e = cudaGetLastError();
+  }
+  return e;
+}
+
+}  // namespace
+
+bool attn_tc_supported(const AttnArgs& a) {
+  if (a.dk != 64 && a.dk != 128) return false;
+  if (a.Tq < 1 || a.Tk < 1 || a.Tq > 8192 || a.Tk > 8192) return false;
+  auto al16 = [](const void* p) { return ((uintptr_t)p & 15) == 0; };
+  if (!al16(a.Q) || !al16(a.K) || !al16(a.V) || !al16(a.O)) return false;
+  if (a.ldq % 8 || a.ldk % 8 || a.ldv % 8 || a.ldo % 8) return false;
+  if (a.causal && a.Tq != a.Tk) return false;
+  return tc::get_encode() != nullptr;
+}
+
+cudaError_t attn_fwd_tc(const AttnArgs& a, int* d_status, cudaStream_t st) {
+  if (a.B == 0) return cudaSuccess;
+  return a.dk == 64 ? fwd_launch<64>(a, d_status, st) : fwd_launch<128>(a, d_status, st);
+}
+
+cudaError_t attn_bwd_tc(const AttnArgs& a, int* d_status, cudaStream_t st) {
+  if (a.B == 0) return cudaSuccess;
+  auto al16 = [](const void* p) { return ((uintptr_t)p & 15) == 0; };
+  if (!al16(a.dO) || !al16(a.dQ) || !al16(a.dK) || !al16(a.dV) || a.lddo % 8 || a.lddq % 8 || a.lddk % 8 ||
+      a.lddv % 8)
+    return cudaErrorInvalidValue;
+  return a.dk == 64 ? bwd_launch<64>(a, d_status, st) : bwd_launch<128>(a, d_status, st);
+}

@@ -90,6 +90,10 @@ struct AttnArgs {
 };
 cudaError_t attn_fwd_simt(int dtype, const AttnArgs& a, cudaStream_t st);
 cudaError_t attn_bwd_simt(int dtype, const AttnArgs& a, cudaStream_t st);
+// tcgen05 path: bf16, d_kv 64 or 128.  The backward also needs O (for delta = rowsum(dO*O)).
+bool attn_tc_supported(const AttnArgs& a);
+cudaError_t attn_fwd_tc(const AttnArgs& a, int* d_status, cudaStream_t st);
+cudaError_t attn_bwd_tc(const AttnArgs& a, int* d_status, cudaStream_t st);
 
 // element-wise / row kernels
 cudaError_t launch_prep(const int* enc_tok, const int* enc_seg, const int* dec_tgt, const int* dec_seg,

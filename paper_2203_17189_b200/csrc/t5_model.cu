@@ -374,7 +374,10 @@ void attn_forward(Ctx& cx, const AttnP& p, const AttnWs& a, float* x_out, const 
   }
   AttnArgs t;
   attn_args(cx, a, gm, cross, &t);
-  CKL(CAT_ATTN_FWD, 1, attn_fwd_simt(dt, t, cx.st), "attn_fwd");
+  if (dt == DT_BF16 && !(c.flags & 1) && attn_tc_supported(t))
+    CKL(CAT_ATTN_FWD, 1, attn_fwd_tc(t, cx.w->status, cx.st), "attn_fwd (tcgen05)");
+  else
+    CKL(CAT_ATTN_FWD, 1, attn_fwd_simt(dt, t, cx.st), "attn_fwd");
   proj_fwd(cx, a.ctx, I, p.o, (int)gm.Nq, d, I, x_out, d, 1.f, a.x, "o proj");
 }
 
@@ -398,7 +401,10 @@ void attn_backward(Ctx& cx, const AttnP& p, const AttnWs& a, float* dX, void* dX
     t.dQ = w.dqkv; t.dK = eoff(cx.h, w.dqkv, I); t.dV = eoff(cx.h, w.dqkv, 2 * I);
     t.lddq = t.lddk = t.lddv = 3 * I;
   }
-  CKL(CAT_ATTN_BWD, 3, attn_bwd_simt(dt, t, cx.st), "attn_bwd");
+  if (dt == DT_BF16 && !(c.flags & 1) && attn_tc_supported(t))
+    CKL(CAT_ATTN_BWD, 3, attn_bwd_tc(t, cx.w->status, cx.st), "attn_bwd (tcgen05)");
+  else
+    CKL(CAT_ATTN_BWD, 3, attn_bwd_simt(dt, t, cx.st), "attn_bwd");
   if (!cross) {
     proj_wgrad(cx, w.dqkv, 3 * I, a.y, d, p.q, Nq, 3 * I, d, 1.f, "wgrad qkv");
     proj_dgrad(cx, w.dqkv, 3 * I, p.q, Nq, 3 * I, d, w.dy, d, 1.f, 0, 0, "dgrad qkv");
@@ -796,6 +802,33 @@ int t5_xent_zloss(int32_t dtype, void* d_logits, const int32_t* d_targets, int32
   if ((dtype != DT_F32 && dtype != DT_BF16) || vocab < 8 || vocab % 8 || n_rows < 0) return T5_ERR_ARG;
   cudaError_t e = launch_xent(dtype, d_logits, d_targets, n_rows, vocab, z_loss, d_W, d_sums, d_lse,
                               (cudaStream_t)stream);
+  return e == cudaSuccess ? T5_OK : T5_ERR_CUDA;
+}
+
+int t5_attention(int32_t dtype, int32_t impl, int32_t backward, int32_t B, int32_t H, int32_t Tq, int32_t Tk,
+                 int32_t d_kv, int32_t causal, float scale, const void* d_q, int32_t ldq, const void* d_k,
+                 int32_t ldk, const void* d_v, int32_t ldv, void* d_o, int32_t ldo, float* d_lse,
+                 const int32_t* d_code_q, const int32_t* d_code_k, const float* d_bias_delta, const void* d_do,
+                 int32_t lddo, void* d_dq, int32_t lddq, void* d_dk, int32_t lddk, void* d_dv, int32_t lddv,
+                 float* d_delta, float* d_dbias_delta, void* stream) {
+  if (!d_q || !d_k || !d_v || !d_o || !d_lse || !d_code_q || !d_code_k) return T5_ERR_NULL;
+  if (backward && (!d_do || !d_dq || !d_dk || !d_dv || !d_delta)) return T5_ERR_NULL;
+  if ((dtype != DT_F32 && dtype != DT_BF16) || B < 0 || H < 1 || Tq < 1 || Tk < 1) return T5_ERR_ARG;
+  if (d_kv != 32 && d_kv != 64 && d_kv != 128) return T5_ERR_ARG;
+  AttnArgs a;
+  memset(&a, 0, sizeof a);
+  a.Q = d_q; a.K = d_k; a.V = d_v; a.O = d_o; a.ldq = ldq; a.ldk = ldk; a.ldv = ldv; a.ldo = ldo; a.lse = d_lse;
+  a.B = B; a.H = H; a.Tq = Tq; a.Tk = Tk; a.dk = d_kv; a.code_q = d_code_q; a.code_k = d_code_k; a.causal = causal;
+  a.bias_delta = d_bias_delta; a.scale = scale; a.dO = d_do; a.lddo = lddo; a.dQ = d_dq; a.dK = d_dk; a.dV = d_dv;
+  a.lddq = lddq; a.lddk = lddk; a.lddv = lddv; a.delta = d_delta; a.dbias_delta = d_dbias_delta;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e;
+  if (impl == 0) {
+    e = backward ? attn_bwd_simt(dtype, a, st) : attn_fwd_simt(dtype, a, st);
+  } else {
+    if (dtype != DT_BF16 || !attn_tc_supported(a)) return T5_ERR_ARG;
+    e = backward ? attn_bwd_tc(a, nullptr, st) : attn_fwd_tc(a, nullptr, st);
+  }
   return e == cudaSuccess ? T5_OK : T5_ERR_CUDA;
 }
 
