@@ -69,8 +69,13 @@ typedef struct {
                                1: bfloat16 parameters/operands, float32 accumulation */
   int32_t recompute;        /* activation policy: 0 keep everything, 1 recompute cheap
                                element-wise pieces in the backward pass */
-  int32_t flags;            /* bit 0: use the plain SIMT GEMM/attention kernels also in
-                               bfloat16 mode (debugging aid) */
+  int32_t flags;            /* debugging aids for bfloat16 mode: bit 0 = use the plain SIMT
+                               GEMM kernel, bit 1 = use the plain SIMT attention kernels.
+                               In float32 mode bits 4..16 round one family of intermediates
+                               to bfloat16 in place (normed activations, projections, context,
+                               FFN pre-activations, gated product, logits, dlogits, residual
+                               gradient copy, dgrad outputs, dcontext, dq/dk/dv, d(gated),
+                               d(pre-activations)) to attribute bfloat16 error */
 } t5_config;
 
 /* One batch.  All pointers are device pointers to int32 arrays. */
@@ -192,14 +197,16 @@ T5_API int t5_gemm(int32_t dtype, int32_t impl, int32_t M, int32_t N, int32_t K,
  * the position codes (and j <= i when causal), P = softmax_j, O = P V,
  * lse = log sum_j exp S.  Rows of q/o/do/dq are (b*Tq + i), rows of k/v/dk/dv
  * are (b*Tk + j); head h occupies columns [h*d_kv, (h+1)*d_kv); ld* are row
- * strides in elements.  d_bias_delta [H, Tq+Tk-1] may be NULL.  Backward writes
+ * strides in elements.  d_bias_delta [H, Tq+Tk-1] may be NULL.  d_o32 (may be
+ * NULL) is a dense float32 [B*Tq, H*d_kv] copy of O that forward writes and
+ * backward reads for delta = rowsum(dO * O).  Backward writes
  * dq, dk, dv, uses d_delta [B,H,Tq] as scratch and ADDS dS summed along
  * diagonals into d_dbias_delta (may be NULL).  impl 0 = SIMT kernels,
  * 1 = tcgen05 kernels (bfloat16, d_kv 64 or 128). */
 T5_API int t5_attention(int32_t dtype, int32_t impl, int32_t backward, int32_t B, int32_t H, int32_t Tq,
                         int32_t Tk, int32_t d_kv, int32_t causal, float scale, const void* d_q, int32_t ldq,
                         const void* d_k, int32_t ldk, const void* d_v, int32_t ldv, void* d_o, int32_t ldo,
-                        float* d_lse, const int32_t* d_code_q, const int32_t* d_code_k,
+                        float* d_o32, float* d_lse, const int32_t* d_code_q, const int32_t* d_code_k,
                         const float* d_bias_delta, const void* d_do, int32_t lddo, void* d_dq, int32_t lddq,
                         void* d_dk, int32_t lddk, void* d_dv, int32_t lddv, float* d_delta,
                         float* d_dbias_delta, void* stream);

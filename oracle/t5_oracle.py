@@ -57,6 +57,9 @@ class T5Config:
     rms_eps: float = 1e-6
     attn_scale: float = 1.0
     logit_scale: float = field(default=-1.0)   # <0 -> d_model ** -0.5
+    operand_bf16: bool = False    # round BOTH operands of every matrix product to bfloat16 first
+                                  # (the "bf16 operands, float32 accumulate" precision the larger
+                                  # workloads are stated in); everything else stays in `dtype`
 
     def __post_init__(self):
         if self.logit_scale < 0:
@@ -114,6 +117,26 @@ def bucket_matrix(tq: int, tk: int, bidirectional: bool, num_buckets: int,
                 lut[r] = relative_position_bucket(r, bidirectional, num_buckets, max_distance)
             out[i, j] = lut[r]
     return out
+
+
+# ----------------------------------------------------------------------------
+# Matrix product with optional bfloat16 operand rounding
+# ----------------------------------------------------------------------------
+def round_bf16(a):
+    """Nearest bfloat16 (ties to even) of each element, returned in a's dtype."""
+    f = np.ascontiguousarray(a, dtype=np.float32)
+    u = f.view(np.uint32)
+    r = ((u >> 16) & 1) + np.uint32(0x7FFF)
+    out = ((u + r) & np.uint32(0xFFFF0000)).astype(np.uint32).view(np.float32)
+    return out.reshape(np.shape(a)).astype(np.asarray(a).dtype)
+
+
+def mm(cfg, a, b):
+    """a @ b; with cfg.operand_bf16 both operands are rounded to bfloat16 and the
+    products are accumulated in the working precision."""
+    if cfg.operand_bf16:
+        return round_bf16(a) @ round_bf16(b)
+    return a @ b
 
 
 # ----------------------------------------------------------------------------
@@ -236,9 +259,9 @@ def _attn_fwd(cfg, p, prefix, x_q, y_kv, table, bidirectional, code_q, code_k, c
     dt = x_q.dtype
     yq, r = rms_norm(x_q, p[prefix + ".norm"], cfg.rms_eps)
     ykv = yq if y_kv is None else y_kv
-    Q = yq @ p[prefix + ".q"]
-    K = ykv @ p[prefix + ".k"]
-    Vv = ykv @ p[prefix + ".v"]
+    Q = mm(cfg, yq, p[prefix + ".q"])
+    K = mm(cfg, ykv, p[prefix + ".k"])
+    Vv = mm(cfg, ykv, p[prefix + ".v"])
     tq, tk = Q.shape[0], K.shape[0]
     mask = attention_mask(code_q, code_k, causal)
     bk = None
@@ -248,12 +271,12 @@ def _attn_fwd(cfg, p, prefix, x_q, y_kv, table, bidirectional, code_q, code_k, c
     C = np.zeros((tq, H * k), dtype=dt)
     for h in range(H):
         sl = slice(h * k, (h + 1) * k)
-        S = dt.type(cfg.attn_scale) * (Q[:, sl] @ K[:, sl].T)
+        S = dt.type(cfg.attn_scale) * mm(cfg, Q[:, sl], K[:, sl].T)
         if table is not None:
             S = S + table[bk, h]
         P[h] = masked_softmax(S, mask)
-        C[:, sl] = P[h] @ Vv[:, sl]
-    out = x_q + C @ p[prefix + ".o"]
+        C[:, sl] = mm(cfg, P[h], Vv[:, sl])
+    out = x_q + mm(cfg, C, p[prefix + ".o"])
     cache = dict(x=x_q, r=r, yq=yq, ykv=ykv, Q=Q, K=K, V=Vv, P=P, C=C, bk=bk,
                  self_attn=(y_kv is None))
     return out, cache
@@ -266,26 +289,26 @@ def _attn_bwd(cfg, p, g, gtable, prefix, dout, c):
     H, k = cfg.n_heads, cfg.d_kv
     dt = dout.dtype
     s = dt.type(cfg.attn_scale)
-    g[prefix + ".o"] += c["C"].T @ dout
-    dC = dout @ p[prefix + ".o"].T
+    g[prefix + ".o"] += mm(cfg, c["C"].T, dout)
+    dC = mm(cfg, dout, p[prefix + ".o"].T)
     dQ = np.zeros_like(c["Q"])
     dK = np.zeros_like(c["K"])
     dV = np.zeros_like(c["V"])
     for h in range(H):
         sl = slice(h * k, (h + 1) * k)
         P = c["P"][h]
-        dP = dC[:, sl] @ c["V"][:, sl].T
-        dV[:, sl] = P.T @ dC[:, sl]
+        dP = mm(cfg, dC[:, sl], c["V"][:, sl].T)
+        dV[:, sl] = mm(cfg, P.T, dC[:, sl])
         dS = P * (dP - np.sum(dP * P, axis=-1, keepdims=True))
         if gtable is not None:
             np.add.at(gtable[:, h], c["bk"].ravel(), dS.ravel())
-        dQ[:, sl] = s * (dS @ c["K"][:, sl])
-        dK[:, sl] = s * (dS.T @ c["Q"][:, sl])
-    g[prefix + ".q"] += c["yq"].T @ dQ
-    g[prefix + ".k"] += c["ykv"].T @ dK
-    g[prefix + ".v"] += c["ykv"].T @ dV
-    dyq = dQ @ p[prefix + ".q"].T
-    dykv = dK @ p[prefix + ".k"].T + dV @ p[prefix + ".v"].T
+        dQ[:, sl] = s * mm(cfg, dS, c["K"][:, sl])
+        dK[:, sl] = s * mm(cfg, dS.T, c["Q"][:, sl])
+    g[prefix + ".q"] += mm(cfg, c["yq"].T, dQ)
+    g[prefix + ".k"] += mm(cfg, c["ykv"].T, dK)
+    g[prefix + ".v"] += mm(cfg, c["ykv"].T, dV)
+    dyq = mm(cfg, dQ, p[prefix + ".q"].T)
+    dykv = mm(cfg, dK, p[prefix + ".k"].T) + mm(cfg, dV, p[prefix + ".v"].T)
     if c["self_attn"]:
         dyq = dyq + dykv
         dykv = None
@@ -296,21 +319,21 @@ def _attn_bwd(cfg, p, g, gtable, prefix, dout, c):
 
 def _ffn_fwd(cfg, p, prefix, x):
     y, r = rms_norm(x, p[prefix + ".norm"], cfg.rms_eps)
-    a = y @ p[prefix + ".wi0"]
-    b = y @ p[prefix + ".wi1"]
+    a = mm(cfg, y, p[prefix + ".wi0"])
+    b = mm(cfg, y, p[prefix + ".wi1"])
     hg = gelu_tanh(a) * b
-    out = x + hg @ p[prefix + ".wo"]
+    out = x + mm(cfg, hg, p[prefix + ".wo"])
     return out, dict(x=x, r=r, y=y, a=a, b=b, hg=hg)
 
 
 def _ffn_bwd(cfg, p, g, prefix, dout, c):
-    g[prefix + ".wo"] += c["hg"].T @ dout
-    dhg = dout @ p[prefix + ".wo"].T
+    g[prefix + ".wo"] += mm(cfg, c["hg"].T, dout)
+    dhg = mm(cfg, dout, p[prefix + ".wo"].T)
     da = dhg * c["b"] * gelu_tanh_grad(c["a"])
     db = dhg * gelu_tanh(c["a"])
-    g[prefix + ".wi0"] += c["y"].T @ da
-    g[prefix + ".wi1"] += c["y"].T @ db
-    dy = da @ p[prefix + ".wi0"].T + db @ p[prefix + ".wi1"].T
+    g[prefix + ".wi0"] += mm(cfg, c["y"].T, da)
+    g[prefix + ".wi1"] += mm(cfg, c["y"].T, db)
+    dy = mm(cfg, da, p[prefix + ".wi0"].T) + mm(cfg, db, p[prefix + ".wi1"].T)
     dxn, dg = rms_norm_bwd(dy, c["x"], p[prefix + ".norm"], c["r"])
     g[prefix + ".norm"] += dg
     return dout + dxn
@@ -351,15 +374,15 @@ def _decoder_fwd(cfg, p, targets_row, dseg_row, enc_y, enc_code):
         x, cf = _ffn_fwd(cfg, p, f"dec.L{l}.ffn", x)
         caches.append((cs, cc, cf))
     z, r = rms_norm(x, p["dec.final_norm"], cfg.rms_eps)
-    logits = x.dtype.type(cfg.logit_scale) * (z @ p["token_embed"].T)
+    logits = x.dtype.type(cfg.logit_scale) * mm(cfg, z, p["token_embed"].T)
     return logits, dict(u=u, layers=caches, x_final=x, r_final=r, z=z)
 
 
 def _decoder_bwd(cfg, p, g, dlogits, c, enc_y):
     dt = dlogits.dtype
     ls = dt.type(cfg.logit_scale)
-    g["token_embed"] += ls * (dlogits.T @ c["z"])
-    dz = ls * (dlogits @ p["token_embed"])
+    g["token_embed"] += ls * mm(cfg, dlogits.T, c["z"])
+    dz = ls * mm(cfg, dlogits, p["token_embed"])
     dx, dg = rms_norm_bwd(dz, c["x_final"], p["dec.final_norm"], c["r_final"])
     g["dec.final_norm"] += dg
     denc = None if enc_y is None else np.zeros_like(enc_y)

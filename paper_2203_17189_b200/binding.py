@@ -82,7 +82,7 @@ def lib():
         L.t5_relpos_buckets.argtypes = [i32, i32, i32, i32, i32, vp, vp]
         L.t5_xent_zloss.argtypes = [i32, vp, vp, i32, i32, f32, vp, vp, vp, vp]
         L.t5_gemm.argtypes = [i32, i32, i32, i32, i32, f32, vp, i32, i32, vp, i32, i32, vp, i32, i32, i32, vp]
-        L.t5_attention.argtypes = ([i32] * 9 + [f32] + [vp, i32] * 3 + [vp, i32, vp, vp, vp, vp]
+        L.t5_attention.argtypes = ([i32] * 9 + [f32] + [vp, i32] * 3 + [vp, i32, vp, vp, vp, vp, vp]
                                    + [vp, i32] * 4 + [vp, vp, vp])
         for n in EXPORTS:
             if n != "t5_last_error":
@@ -243,13 +243,13 @@ def t5_gemm(impl, M, N, K, alpha, A, lda, a_kmajor, B, ldb, b_kmajor, D, ldd, ac
 
 
 def t5_attention(impl, backward, B, H, Tq, Tk, d_kv, causal, scale, q, k, v, o, lse, code_q, code_k, bias_delta,
-                 do=None, dq=None, dk=None, dv=None, delta=None, dbias_delta=None):
+                 do=None, dq=None, dk=None, dv=None, delta=None, dbias_delta=None, o32=None):
     """q/k/v/o/do/dq/dk/dv: 2-D tensors (possibly column-sliced views) with rows = tokens."""
     dtype = 0 if q.dtype == torch.float32 else 1
 
     def ld(t):
         return 0 if t is None else t.stride(0)
     _check(lib().t5_attention(dtype, impl, int(backward), B, H, Tq, Tk, d_kv, int(causal), scale,
-                              _ptr(q), ld(q), _ptr(k), ld(k), _ptr(v), ld(v), _ptr(o), ld(o), _ptr(lse),
+                              _ptr(q), ld(q), _ptr(k), ld(k), _ptr(v), ld(v), _ptr(o), ld(o), _ptr(o32), _ptr(lse),
                               _ptr(code_q), _ptr(code_k), _ptr(bias_delta), _ptr(do), ld(do), _ptr(dq), ld(dq),
                               _ptr(dk), ld(dk), _ptr(dv), ld(dv), _ptr(delta), _ptr(dbias_delta), _stream()))

@@ -26,7 +26,8 @@ struct P {   // plain-pointer copy of AttnArgs for the kernels
   const void *Q, *K, *V, *dO;
   void *O, *dQ, *dK, *dV;
   int ldq, ldk, ldv, ldo, lddo, lddq, lddk, lddv;
-  float *lse, *delta, *dbias_delta;
+  float *lse, *delta, *dbias_delta, *O32;
+  int ldo32;
   const float* bias_delta;
   const int *code_q, *code_k;
   int B, H, Tq, Tk, causal;
@@ -106,6 +107,9 @@ __global__ void __launch_bounds__(128) attn_fwd_kernel(P a) {
 #pragma unroll
     for (int c = 0; c < C; ++c)
       O[(int64_t)(b * a.Tq + i) * a.ldo + h * DK + lane + 32 * c] = from_f<T>(o[qq][c] * inv);
+    if (a.O32)
+#pragma unroll
+      for (int c = 0; c < C; ++c) a.O32[(int64_t)(b * a.Tq + i) * a.ldo32 + h * DK + lane + 32 * c] = o[qq][c] * inv;
     if (lane == 0) a.lse[(int64_t)(b * a.H + h) * a.Tq + i] = l[qq] > 0.f ? m[qq] + logf(l[qq]) : -INFINITY;
   }
 }
@@ -122,7 +126,8 @@ __global__ void attn_delta_kernel(P a) {
   float s = 0.f;
 #pragma unroll
   for (int c = 0; c < DK / 32; ++c)
-    s += to_f(O[(int64_t)row * a.ldo + h * DK + lane + 32 * c]) *
+    s += (a.O32 ? a.O32[(int64_t)row * a.ldo32 + h * DK + lane + 32 * c]
+                : to_f(O[(int64_t)row * a.ldo + h * DK + lane + 32 * c])) *
          to_f(dO[(int64_t)row * a.lddo + h * DK + lane + 32 * c]);
   s = wsum(s);
   if (lane == 0) a.delta[(int64_t)(b * a.H + h) * a.Tq + i] = s;
@@ -317,6 +322,7 @@ P to_p(const AttnArgs& a) {
   p.Q = a.Q; p.K = a.K; p.V = a.V; p.dO = a.dO; p.O = a.O; p.dQ = a.dQ; p.dK = a.dK; p.dV = a.dV;
   p.ldq = a.ldq; p.ldk = a.ldk; p.ldv = a.ldv; p.ldo = a.ldo; p.lddo = a.lddo; p.lddq = a.lddq;
   p.lddk = a.lddk; p.lddv = a.lddv; p.lse = a.lse; p.delta = a.delta; p.dbias_delta = a.dbias_delta;
+  p.O32 = a.O32; p.ldo32 = a.ldo32;
   p.bias_delta = a.bias_delta; p.code_q = a.code_q; p.code_k = a.code_k; p.B = a.B; p.H = a.H;
   p.Tq = a.Tq; p.Tk = a.Tk; p.causal = a.causal; p.scale = a.scale;
   return p;

@@ -29,7 +29,8 @@ using namespace tc;
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct TcParams {
-  const void* O;        // forward: output (written); backward: unused
+  float* o32;           // forward: optional float32 copy of the output rows
+  int ldo32;
   void* out0;           // forward: O; dQ kernel: dQ; dKV kernel: dK
   void* out1;           // dKV kernel: dV
   int ld0, ld1;
@@ -201,7 +202,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
         int ck = codes_s[j];
         bool valid = ck != 0 && ck == cq && (!p.causal || j <= i);
         float s = __uint_as_float(r[jj]) * sc2 + bias_s[j - tid + 127];
-        float e = valid ? exp2f(s - m_new) : 0.f;
+        // the row sum uses the bf16-rounded probabilities, so the weights the MMA applies sum to one
+        float e = valid ? __bfloat162float(__float2bfloat16_rn(exp2f(s - m_new))) : 0.f;
         pv[jj] = e;
         lsum += e;
       }
@@ -266,6 +268,12 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
       v.z = pack_bf16(o[d + 4] * inv, o[d + 5] * inv);
       v.w = pack_bf16(o[d + 6] * inv, o[d + 7] * inv);
       *reinterpret_cast<uint4*>(orow + d) = v;
+    }
+    if (p.o32) {
+      float* o32 = p.o32 + (int64_t)(b * p.Tq + i) * p.ldo32 + h * DK;
+#pragma unroll
+      for (int d = 0; d < DK; d += 4)
+        *reinterpret_cast<float4*>(o32 + d) = make_float4(o[d] * inv, o[d + 1] * inv, o[d + 2] * inv, o[d + 3] * inv);
     }
     // natural-log log-sum-exp of the (unscaled-by-log2e) scores
     p.lse[(int64_t)(b * p.H + h) * p.Tq + i] = l_run > 0.f ? (m_run + log2f(l_run)) / kLog2e : -INFINITY;
@@ -705,8 +713,9 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
 
 // ----------------------------------------------------------------------------- delta = rowsum(dO * O)
 template <int DK>
-__global__ void attn_delta_tc_kernel(const bf16* __restrict__ O, int ldo, const bf16* __restrict__ dO, int lddo,
-                                     float* __restrict__ delta, int B, int H, int Tq) {
+__global__ void attn_delta_tc_kernel(const bf16* __restrict__ O, int ldo, const float* __restrict__ O32, int ldo32,
+                                     const bf16* __restrict__ dO, int lddo, float* __restrict__ delta, int B, int H,
+                                     int Tq) {
   int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (gw >= B * Tq * H) return;
   int h = gw % H, row = gw / H;
@@ -714,9 +723,14 @@ __global__ void attn_delta_tc_kernel(const bf16* __restrict__ O, int ldo, const 
   float s = 0.f;
 #pragma unroll
   for (int c = 0; c < DK / 64; ++c) {
-    __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(O + (int64_t)row * ldo + h * DK + c * 64 + lane * 2);
-    __nv_bfloat162 g = *reinterpret_cast<const __nv_bfloat162*>(dO + (int64_t)row * lddo + h * DK + c * 64 + lane * 2);
-    float2 fa = __bfloat1622float2(a), fg = __bfloat1622float2(g);
+    int col = h * DK + c * 64 + lane * 2;
+    __nv_bfloat162 g = *reinterpret_cast<const __nv_bfloat162*>(dO + (int64_t)row * lddo + col);
+    float2 fg = __bfloat1622float2(g), fa;
+    if (O32) {
+      fa = *reinterpret_cast<const float2*>(O32 + (int64_t)row * ldo32 + col);
+    } else {
+      fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(O + (int64_t)row * ldo + col));
+    }
     s += fa.x * fg.x + fa.y * fg.y;
   }
 #pragma unroll
@@ -757,7 +771,7 @@ cudaError_t fwd_launch(const AttnArgs& a, int* status, cudaStream_t st) {
   cudaError_t e = cudaFuncSetAttribute(attn_fwd_tc_kernel<DK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   TcParams p = base_params(a, status);
-  p.out0 = a.O; p.ld0 = a.ldo;
+  p.out0 = a.O; p.ld0 = a.ldo; p.o32 = a.O32; p.ldo32 = a.ldo32;
   dim3 grid((a.Tq + 127) / 128, a.H, a.B);
   attn_fwd_tc_kernel<DK><<<grid, 128, smem, st>>>(mq, mk, mv, p);
   return cudaGetLastError();
@@ -767,8 +781,8 @@ template <int DK>
 cudaError_t bwd_launch(const AttnArgs& a, int* status, cudaStream_t st) {
   int I = a.H * DK;
   int warps = a.B * a.Tq * a.H;
-  attn_delta_tc_kernel<DK><<<(warps + 7) / 8, 256, 0, st>>>((const bf16*)a.O, a.ldo, (const bf16*)a.dO, a.lddo,
-                                                            a.delta, a.B, a.H, a.Tq);
+  attn_delta_tc_kernel<DK><<<(warps + 7) / 8, 256, 0, st>>>((const bf16*)a.O, a.ldo, a.O32, a.ldo32,
+                                                            (const bf16*)a.dO, a.lddo, a.delta, a.B, a.H, a.Tq);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   TcParams p = base_params(a, status);
@@ -810,6 +824,7 @@ bool attn_tc_supported(const AttnArgs& a) {
   auto al16 = [](const void* p) { return ((uintptr_t)p & 15) == 0; };
   if (!al16(a.Q) || !al16(a.K) || !al16(a.V) || !al16(a.O)) return false;
   if (a.ldq % 8 || a.ldk % 8 || a.ldv % 8 || a.ldo % 8) return false;
+  if (a.O32 && (!al16(a.O32) || a.ldo32 % 4)) return false;
   if (a.causal && a.Tq != a.Tk) return false;
   return tc::get_encode() != nullptr;
 }

@@ -76,6 +76,9 @@ struct AttnArgs {
   void* O;
   int ldq, ldk, ldv, ldo;
   float* lse;               // [B,H,Tq]
+  float* O32; int ldo32;    // optional float32 copy of O (written by forward, read by backward): delta =
+                            // rowsum(dO * O) must see O unrounded, or a component shared by all values
+                            // of a row no longer cancels in dS = P (dP - delta)
   int B, H, Tq, Tk, dk;
   const int* code_q;        // [B,Tq]
   const int* code_k;        // [B,Tk]
@@ -119,6 +122,7 @@ cudaError_t launch_xent(int dtype, void* logits, const int* targets, int rows, i
 cudaError_t launch_finalize_loss(const double* sums, const float* W, float* loss4, cudaStream_t st);
 cudaError_t launch_fill_normal(int dtype, void* p, int64_t n, int64_t flat_offset, uint64_t seed,
                                float stddev, float mean, cudaStream_t st);
+cudaError_t launch_round_bf16(float* p, int64_t n, cudaStream_t st);   // in place: float -> nearest bf16 -> float
 cudaError_t launch_cast_f32_to(int dtype, const float* src, void* dst, int64_t n, cudaStream_t st);
 // bias tables
 cudaError_t launch_relbias_expand(int dtype, const BucketSpec& spec, const void* table, int H, int Tq,

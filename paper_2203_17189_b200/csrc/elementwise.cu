@@ -358,6 +358,11 @@ __global__ void cast_kernel(const float* __restrict__ s, T* __restrict__ d, int6
   }
 }
 
+__global__ void round_bf16_kernel(float* p, int64_t n) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) p[i] = __bfloat162float(__float2bfloat16_rn(p[i]));
+}
+
 inline unsigned blocks_for(int64_t n, int per) { return (unsigned)((n + per - 1) / per); }
 
 }  // namespace
@@ -503,5 +508,11 @@ cudaError_t launch_cast_f32_to(int dtype, const float* src, void* dst, int64_t n
     cast_kernel<float><<<blocks_for(n, 1024), 256, 0, st>>>(src, (float*)dst, n);
   else
     cast_kernel<bf16><<<blocks_for(n, 1024), 256, 0, st>>>(src, (bf16*)dst, n);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_round_bf16(float* p, int64_t n, cudaStream_t st) {
+  if (n == 0) return cudaSuccess;
+  round_bf16_kernel<<<blocks_for(n, 256), 256, 0, st>>>(p, n);
   return cudaGetLastError();
 }

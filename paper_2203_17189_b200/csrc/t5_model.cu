@@ -27,7 +27,7 @@ struct EncLayerP { AttnP attn; FfnP ffn; };
 struct DecLayerP { AttnP self, cross; FfnP ffn; };
 
 // per-sub-layer saved activations
-struct AttnWs { float* x; void* y; float* rstd; void* q; void* kv; void* ctx; float* lse; };
+struct AttnWs { float* x; void* y; float* rstd; void* q; void* kv; void* ctx; float* ctx32; float* lse; };
 struct FfnWs { float* x; void* y; float* rstd; void* h; void* hg; };
 
 struct Workspace {
@@ -176,6 +176,7 @@ void plan_workspace(const t5_handle* h, int B, int Te, int Td, char* base, Works
     a.q = take(Nq * (cross ? I : 3 * I) * es);
     a.kv = cross ? take(Nk * 2 * I * es) : nullptr;
     a.ctx = take(Nq * I * es);
+    a.ctx32 = es == 2 ? (float*)take(Nq * I * 4) : nullptr;   // unrounded copy for the backward's delta
     a.lse = (float*)take((int64_t)B * H * Tq * 4);
     return a;
   };
@@ -302,6 +303,14 @@ void gemm(Ctx& cx, const GemmArgs& g, const char* what) {
   }
 }
 
+// Numerics debugging aid: in float32 mode, flag bit `bit` rounds one family of intermediates to
+// bfloat16 precision in place, to attribute the bfloat16 mode's error to the buffer that causes it.
+enum { RB_Y = 4, RB_QKV, RB_CTX, RB_H, RB_HG, RB_LOGITS, RB_DLOGITS, RB_DXB, RB_DY, RB_DCTX, RB_DQKV, RB_DHG, RB_DH };
+void dbg_round(Ctx& cx, void* p, int64_t n, int bit) {
+  if (cx.h->cfg.dtype != DT_F32 || !((cx.h->cfg.flags >> bit) & 1)) return;
+  CK(launch_round_bf16((float*)p, n, cx.st), "debug rounding");
+}
+
 // Y[M,N] = alpha X[M,K] W[N,K]^T (+ resid)
 void proj_fwd(Ctx& cx, const void* X, int ldx, int64_t w_off, int M, int N, int K, void* Y, int ldy, float alpha,
               const float* resid, const char* what) {
@@ -353,7 +362,7 @@ void attn_args(Ctx& cx, const AttnWs& a, const AttnGeom& gm, bool cross, AttnArg
   } else {
     t.Q = a.q; t.K = eoff(cx.h, a.q, I); t.V = eoff(cx.h, a.q, 2 * I); t.ldq = t.ldk = t.ldv = 3 * I;
   }
-  t.O = a.ctx; t.ldo = I; t.lse = a.lse;
+  t.O = a.ctx; t.ldo = I; t.lse = a.lse; t.O32 = a.ctx32; t.ldo32 = I;
   t.B = cx.B; t.H = c.n_heads; t.Tq = gm.Tq; t.Tk = gm.Tk; t.dk = c.d_kv;
   t.code_q = gm.code_q; t.code_k = gm.code_k; t.causal = gm.causal;
   t.bias_delta = gm.bias; t.scale = c.attn_scale;
@@ -366,18 +375,23 @@ void attn_forward(Ctx& cx, const AttnP& p, const AttnWs& a, float* x_out, const 
   bool cross = kv_src != nullptr;
   CKL(CAT_NORM, 1, launch_rmsnorm_fwd(dt, a.x, pptr(cx.h, cx.params, p.norm), a.y, a.rstd, (int)gm.Nq, d, c.rms_eps, cx.st),
      "rmsnorm_fwd");
+  dbg_round(cx, a.y, gm.Nq * d, RB_Y);
   if (!cross) {
     proj_fwd(cx, a.y, d, p.q, (int)gm.Nq, 3 * I, d, a.q, 3 * I, 1.f, nullptr, "qkv proj");
+    dbg_round(cx, a.q, gm.Nq * 3 * I, RB_QKV);
   } else {
     proj_fwd(cx, a.y, d, p.q, (int)gm.Nq, I, d, a.q, I, 1.f, nullptr, "q proj");
     proj_fwd(cx, kv_src, d, p.k, (int)gm.Nk, 2 * I, d, a.kv, 2 * I, 1.f, nullptr, "kv proj");
+    dbg_round(cx, a.q, gm.Nq * I, RB_QKV);
+    dbg_round(cx, a.kv, gm.Nk * 2 * I, RB_QKV);
   }
   AttnArgs t;
   attn_args(cx, a, gm, cross, &t);
-  if (dt == DT_BF16 && !(c.flags & 1) && attn_tc_supported(t))
+  if (dt == DT_BF16 && !(c.flags & 2) && attn_tc_supported(t))
     CKL(CAT_ATTN_FWD, 1, attn_fwd_tc(t, cx.w->status, cx.st), "attn_fwd (tcgen05)");
   else
     CKL(CAT_ATTN_FWD, 1, attn_fwd_simt(dt, t, cx.st), "attn_fwd");
+  dbg_round(cx, a.ctx, gm.Nq * I, RB_CTX);
   proj_fwd(cx, a.ctx, I, p.o, (int)gm.Nq, d, I, x_out, d, 1.f, a.x, "o proj");
 }
 
@@ -391,6 +405,7 @@ void attn_backward(Ctx& cx, const AttnP& p, const AttnWs& a, float* dX, void* dX
   int Nq = (int)gm.Nq, Nk = (int)gm.Nk;
   proj_wgrad(cx, dXb, d, a.ctx, I, p.o, Nq, d, I, 1.f, "wgrad o");
   proj_dgrad(cx, dXb, d, p.o, Nq, d, I, w.dctx, I, 1.f, 0, 0, "dgrad o");
+  dbg_round(cx, w.dctx, (int64_t)Nq * I, RB_DCTX);
   AttnArgs t;
   attn_args(cx, a, gm, cross, &t);
   t.dO = w.dctx; t.lddo = I; t.delta = w.delta; t.dbias_delta = gm.dbias;
@@ -401,10 +416,12 @@ void attn_backward(Ctx& cx, const AttnP& p, const AttnWs& a, float* dX, void* dX
     t.dQ = w.dqkv; t.dK = eoff(cx.h, w.dqkv, I); t.dV = eoff(cx.h, w.dqkv, 2 * I);
     t.lddq = t.lddk = t.lddv = 3 * I;
   }
-  if (dt == DT_BF16 && !(c.flags & 1) && attn_tc_supported(t))
+  if (dt == DT_BF16 && !(c.flags & 2) && attn_tc_supported(t))
     CKL(CAT_ATTN_BWD, 3, attn_bwd_tc(t, cx.w->status, cx.st), "attn_bwd (tcgen05)");
   else
     CKL(CAT_ATTN_BWD, 3, attn_bwd_simt(dt, t, cx.st), "attn_bwd");
+  dbg_round(cx, w.dqkv, (int64_t)Nq * (cross ? I : 3 * I), RB_DQKV);
+  if (cross) dbg_round(cx, w.dkv, (int64_t)Nk * 2 * I, RB_DQKV);
   if (!cross) {
     proj_wgrad(cx, w.dqkv, 3 * I, a.y, d, p.q, Nq, 3 * I, d, 1.f, "wgrad qkv");
     proj_dgrad(cx, w.dqkv, 3 * I, p.q, Nq, 3 * I, d, w.dy, d, 1.f, 0, 0, "dgrad qkv");
@@ -414,9 +431,11 @@ void attn_backward(Ctx& cx, const AttnP& p, const AttnWs& a, float* dX, void* dX
     proj_wgrad(cx, w.dkv, 2 * I, kv_src, d, p.k, Nk, 2 * I, d, 1.f, "wgrad kv");
     proj_dgrad(cx, w.dkv, 2 * I, p.k, Nk, 2 * I, d, dY32, d, 1.f, 1, dY_accumulate, "dgrad kv");
   }
+  dbg_round(cx, w.dy, (int64_t)Nq * d, RB_DY);
   CKL(CAT_NORM, 2, launch_rmsnorm_bwd(dt, w.dy, 0, a.x, a.rstd, pptr(cx.h, cx.params, p.norm), dX, dX, dXb, cx.grads + p.norm,
                         w.norm_partial, Nq, d, cx.st),
      "rmsnorm_bwd");
+  dbg_round(cx, dXb, (int64_t)Nq * d, RB_DXB);
 }
 
 void ffn_forward(Ctx& cx, const FfnP& p, const FfnWs& f, float* x_out, int64_t N) {
@@ -424,8 +443,11 @@ void ffn_forward(Ctx& cx, const FfnP& p, const FfnWs& f, float* x_out, int64_t N
   int d = c.d_model, F = c.d_ff, dt = c.dtype;
   CKL(CAT_NORM, 1, launch_rmsnorm_fwd(dt, f.x, pptr(cx.h, cx.params, p.norm), f.y, f.rstd, (int)N, d, c.rms_eps, cx.st),
      "rmsnorm_fwd");
+  dbg_round(cx, f.y, N * d, RB_Y);
   proj_fwd(cx, f.y, d, p.wi0, (int)N, 2 * F, d, f.h, 2 * F, 1.f, nullptr, "wi proj");
+  dbg_round(cx, f.h, N * 2 * F, RB_H);
   CKL(CAT_GEGLU, 1, launch_geglu_fwd(dt, f.h, f.hg, (int)N, F, cx.st), "geglu_fwd");
+  dbg_round(cx, f.hg, N * F, RB_HG);
   proj_fwd(cx, f.hg, F, p.wo, (int)N, d, F, x_out, d, 1.f, f.x, "wo proj");
 }
 
@@ -435,12 +457,16 @@ void ffn_backward(Ctx& cx, const FfnP& p, const FfnWs& f, float* dX, void* dXb, 
   int d = c.d_model, F = c.d_ff, dt = c.dtype, n = (int)N;
   proj_wgrad(cx, dXb, d, f.hg, F, p.wo, n, d, F, 1.f, "wgrad ffn.wo");
   proj_dgrad(cx, dXb, d, p.wo, n, d, F, w.dhg, F, 1.f, 0, 0, "dgrad ffn.wo");
+  dbg_round(cx, w.dhg, N * F, RB_DHG);
   CKL(CAT_GEGLU, 1, launch_geglu_bwd(dt, w.dhg, f.h, w.dh, n, F, cx.st), "geglu_bwd");
+  dbg_round(cx, w.dh, N * 2 * F, RB_DH);
   proj_wgrad(cx, w.dh, 2 * F, f.y, d, p.wi0, n, 2 * F, d, 1.f, "wgrad ffn.wi");
   proj_dgrad(cx, w.dh, 2 * F, p.wi0, n, 2 * F, d, w.dy, d, 1.f, 0, 0, "dgrad ffn.wi");
+  dbg_round(cx, w.dy, N * d, RB_DY);
   CKL(CAT_NORM, 2, launch_rmsnorm_bwd(dt, w.dy, 0, f.x, f.rstd, pptr(cx.h, cx.params, p.norm), dX, dX, dXb, cx.grads + p.norm,
                         w.norm_partial, n, d, cx.st),
      "rmsnorm_bwd");
+  dbg_round(cx, dXb, N * d, RB_DXB);
 }
 
 AttnGeom enc_geom(Ctx& cx) {
@@ -495,6 +521,7 @@ void encoder_forward(Ctx& cx, const t5_batch* b) {
   CKL(CAT_NORM, 1, launch_rmsnorm_fwd(c.dtype, w.enc_x_final, pptr(cx.h, cx.params, cx.h->enc_final_norm), w.enc_out,
                         w.enc_rstd_f, (int)Ne, d, c.rms_eps, cx.st),
      "enc final norm");
+  dbg_round(cx, w.enc_out, Ne * d, RB_Y);
 }
 
 // enc_y: encoder output used by cross-attention (NULL for decoder-only); logits_out: where logits go
@@ -518,8 +545,10 @@ void decoder_forward(Ctx& cx, const void* enc_y, void* logits_out) {
   CKL(CAT_NORM, 1, launch_rmsnorm_fwd(c.dtype, w.dec_x_final, pptr(cx.h, cx.params, cx.h->dec_final_norm), w.dec_z, w.dec_rstd_f,
                         (int)Nd, d, c.rms_eps, cx.st),
      "dec final norm");
+  dbg_round(cx, w.dec_z, Nd * d, RB_Y);
   proj_fwd(cx, w.dec_z, d, cx.h->token_embed, (int)Nd, c.vocab, d, logits_out, c.vocab, c.logit_scale, nullptr,
            "logits");
+  dbg_round(cx, logits_out, Nd * c.vocab, RB_LOGITS);
 }
 
 void backward(Ctx& cx, const t5_batch* b) {
@@ -535,10 +564,12 @@ void backward(Ctx& cx, const t5_batch* b) {
   // tied embedding: dE = logit_scale dlogits^T Z (overwrites), dZ = logit_scale dlogits E
   proj_wgrad(cx, w.logits, V, w.dec_z, d, cx.h->token_embed, (int)Nd, V, d, c.logit_scale, "wgrad logits");
   proj_dgrad(cx, w.logits, V, cx.h->token_embed, (int)Nd, V, d, w.dy, d, c.logit_scale, 0, 0, "dgrad logits");
+  dbg_round(cx, w.dy, Nd * d, RB_DY);
   CKL(CAT_NORM, 2, launch_rmsnorm_bwd(dt, w.dy, 0, w.dec_x_final, w.dec_rstd_f, pptr(cx.h, cx.params, cx.h->dec_final_norm),
                         nullptr, w.dX_dec, w.dXb_dec, cx.grads + cx.h->dec_final_norm, w.norm_partial, (int)Nd, d,
                         cx.st),
      "dec final norm bwd");
+  dbg_round(cx, w.dXb_dec, Nd * d, RB_DXB);
   AttnGeom gs = self_geom(cx), gc = cross_geom(cx);
   bool first_cross = true;
   for (int l = c.n_dec_layers - 1; l >= 0; --l) {
@@ -560,6 +591,7 @@ void backward(Ctx& cx, const t5_batch* b) {
                         nullptr, w.dX_enc, w.dXb_enc, cx.grads + cx.h->enc_final_norm, w.norm_partial, (int)Ne, d,
                         cx.st),
      "enc final norm bwd");
+  dbg_round(cx, w.dXb_enc, Ne * d, RB_DXB);
   AttnGeom ge = enc_geom(cx);
   for (int l = c.n_enc_layers - 1; l >= 0; --l) {
     ffn_backward(cx, cx.h->enc[l].ffn, w.enc_ffn[l], w.dX_enc, w.dXb_enc, Ne);
@@ -714,6 +746,7 @@ int t5_train_step_fwd_bwd(t5_handle* h, const void* d_params, const t5_batch* ba
                  cx.st),
      "xent");
   CKL(CAT_MISC, 1, launch_finalize_loss(w.sums, w.W_f, d_loss4, cx.st), "finalize loss");
+  dbg_round(cx, w.logits, (int64_t)cx.B * cx.Td * c.vocab, RB_DLOGITS);
   backward(cx, batch);
   return end_call(h, cx);
 }
@@ -807,7 +840,7 @@ int t5_xent_zloss(int32_t dtype, void* d_logits, const int32_t* d_targets, int32
 
 int t5_attention(int32_t dtype, int32_t impl, int32_t backward, int32_t B, int32_t H, int32_t Tq, int32_t Tk,
                  int32_t d_kv, int32_t causal, float scale, const void* d_q, int32_t ldq, const void* d_k,
-                 int32_t ldk, const void* d_v, int32_t ldv, void* d_o, int32_t ldo, float* d_lse,
+                 int32_t ldk, const void* d_v, int32_t ldv, void* d_o, int32_t ldo, float* d_o32, float* d_lse,
                  const int32_t* d_code_q, const int32_t* d_code_k, const float* d_bias_delta, const void* d_do,
                  int32_t lddo, void* d_dq, int32_t lddq, void* d_dk, int32_t lddk, void* d_dv, int32_t lddv,
                  float* d_delta, float* d_dbias_delta, void* stream) {
@@ -817,6 +850,7 @@ int t5_attention(int32_t dtype, int32_t impl, int32_t backward, int32_t B, int32
   if (d_kv != 32 && d_kv != 64 && d_kv != 128) return T5_ERR_ARG;
   AttnArgs a;
   memset(&a, 0, sizeof a);
+  a.O32 = d_o32; a.ldo32 = H * d_kv;
   a.Q = d_q; a.K = d_k; a.V = d_v; a.O = d_o; a.ldq = ldq; a.ldk = ldk; a.ldv = ldv; a.ldo = ldo; a.lse = d_lse;
   a.B = B; a.H = H; a.Tq = Tq; a.Tk = Tk; a.dk = d_kv; a.code_q = d_code_q; a.code_k = d_code_k; a.causal = causal;
   a.bias_delta = d_bias_delta; a.scale = scale; a.dO = d_do; a.lddo = lddo; a.dQ = d_dq; a.dK = d_dk; a.dV = d_dv;

@@ -108,9 +108,10 @@ def test_attention_forward_backward(impl, B, H, Tq, Tk, dk, causal, use_bias, mo
     cq_d = torch.from_numpy(code_q).to(DEV)
     ck_d = torch.from_numpy(code_k).to(DEV)
     bias_d = None if bias is None else torch.from_numpy(bias).to(DEV)
-    Bd.t5_attention(impl, False, B, H, Tq, Tk, dk, causal, scale, q, k, v, o, lse, cq_d, ck_d, bias_d)
+    o32 = torch.full((B * Tq, I), float("nan"), dtype=torch.float32, device=DEV) if B != 3 else None
+    Bd.t5_attention(impl, False, B, H, Tq, Tk, dk, causal, scale, q, k, v, o, lse, cq_d, ck_d, bias_d, o32=o32)
     Bd.t5_attention(impl, True, B, H, Tq, Tk, dk, causal, scale, q, k, v, o, lse, cq_d, ck_d, bias_d,
-                    do=do, dq=dq, dk=dk_t, dv=dv_t, delta=delta, dbias_delta=dbias)
+                    do=do, dq=dq, dk=dk_t, dv=dv_t, delta=delta, dbias_delta=dbias, o32=o32)
     torch.cuda.synchronize()
 
     f64 = lambda t, T: t.float().cpu().numpy().astype(np.float64).reshape(B, T, I)
