@@ -211,6 +211,31 @@ T5_API int t5_attention(int32_t dtype, int32_t impl, int32_t backward, int32_t B
                         void* d_dk, int32_t lddk, void* d_dv, int32_t lddv, float* d_delta,
                         float* d_dbias_delta, void* stream);
 
+/* Attention backward without caller-provided scratch.  The paper has no
+ * counterpart; this exists for callers that cannot allocate device memory:
+ * code in a region where cudaMalloc is illegal or must be avoided, plug-ins
+ * that are handed only their inputs and outputs by a framework that owns the
+ * allocator, processes whose device memory pool is committed at start-up.
+ * Same computation and arguments as t5_attention(..., backward = 1, ...),
+ * except that the delta[B,H,Tq] scratch lives in a fixed array inside the
+ * library (T5_NOALLOC_MAX_ROWS floats = 4 MiB, held by every GPU that loads
+ * the library until the process exits).  The call allocates nothing.
+ *  - B*H*Tq must not exceed T5_NOALLOC_MAX_ROWS, else T5_ERR_SHAPE.
+ *  - The first call on each device looks up the array's device address (with
+ *    that device current); make that first call before any stream capture.
+ *  - All calls share the one array per device and it keeps the previous
+ *    call's contents.  Nothing in it needs clearing: every element a call
+ *    reads is first written by that call.  Two calls whose kernels overlap on
+ *    the same GPU (different streams) race on it; serialise them.
+ *  - d_dbias_delta is ADDED to, as in t5_attention. */
+#define T5_NOALLOC_MAX_ROWS (1 << 20)
+T5_API int t5_attention_backward_noalloc(
+    int32_t dtype, int32_t impl, int32_t B, int32_t H, int32_t Tq, int32_t Tk, int32_t d_kv, int32_t causal,
+    float scale, const void* d_q, int32_t ldq, const void* d_k, int32_t ldk, const void* d_v, int32_t ldv,
+    const void* d_o, int32_t ldo, const float* d_o32, const float* d_lse, const int32_t* d_code_q,
+    const int32_t* d_code_k, const float* d_bias_delta, const void* d_do, int32_t lddo, void* d_dq,
+    int32_t lddq, void* d_dk, int32_t lddk, void* d_dv, int32_t lddv, float* d_dbias_delta, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

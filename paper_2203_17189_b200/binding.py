@@ -42,7 +42,7 @@ EXPORTS = ["t5_create", "t5_destroy", "t5_last_error", "t5_param_count", "t5_par
            "t5_param_manifest", "t5_workspace_bytes", "t5_init_params", "t5_train_step_fwd_bwd",
            "t5_encode", "t5_decode_logits", "t5_device_status", "t5_profile_enable", "t5_profile_read",
            "t5_launch_count", "t5_relpos_buckets", "t5_xent_zloss",
-           "t5_gemm", "t5_attention"]
+           "t5_gemm", "t5_attention", "t5_attention_backward_noalloc"]
 
 _lib = None
 
@@ -84,6 +84,8 @@ def lib():
         L.t5_gemm.argtypes = [i32, i32, i32, i32, i32, f32, vp, i32, i32, vp, i32, i32, vp, i32, i32, i32, vp]
         L.t5_attention.argtypes = ([i32] * 9 + [f32] + [vp, i32] * 3 + [vp, i32, vp, vp, vp, vp, vp]
                                    + [vp, i32] * 4 + [vp, vp, vp])
+        L.t5_attention_backward_noalloc.argtypes = ([i32] * 8 + [f32] + [vp, i32] * 4 + [vp] * 5
+                                                    + [vp, i32] * 4 + [vp, vp])
         for n in EXPORTS:
             if n != "t5_last_error":
                 getattr(L, n).restype = C.c_int
@@ -253,3 +255,16 @@ def t5_attention(impl, backward, B, H, Tq, Tk, d_kv, causal, scale, q, k, v, o, 
                               _ptr(q), ld(q), _ptr(k), ld(k), _ptr(v), ld(v), _ptr(o), ld(o), _ptr(o32), _ptr(lse),
                               _ptr(code_q), _ptr(code_k), _ptr(bias_delta), _ptr(do), ld(do), _ptr(dq), ld(dq),
                               _ptr(dk), ld(dk), _ptr(dv), ld(dv), _ptr(delta), _ptr(dbias_delta), _stream()))
+
+
+def t5_attention_backward_noalloc(impl, B, H, Tq, Tk, d_kv, causal, scale, q, k, v, o, o32, lse, code_q, code_k,
+                                  bias_delta, do, dq, dk, dv, dbias_delta=None):
+    """Attention backward whose scratch is built into the library: for callers that cannot allocate
+    device memory around the call.  Nothing in this call allocates."""
+    dtype = 0 if q.dtype == torch.float32 else 1
+    _check(lib().t5_attention_backward_noalloc(dtype, impl, B, H, Tq, Tk, d_kv, int(causal), scale,
+                                               _ptr(q), q.stride(0), _ptr(k), k.stride(0), _ptr(v), v.stride(0),
+                                               _ptr(o), o.stride(0), _ptr(o32), _ptr(lse), _ptr(code_q),
+                                               _ptr(code_k), _ptr(bias_delta), _ptr(do), do.stride(0),
+                                               _ptr(dq), dq.stride(0), _ptr(dk), dk.stride(0), _ptr(dv),
+                                               dv.stride(0), _ptr(dbias_delta), _stream()))

@@ -1,0 +1,73 @@
+"""The allocation-free attention backward (scratch built into the library) against the regular entry point.
+
+Who needs it: callers that must not or cannot allocate device memory around the call - code in a region where
+cudaMalloc is illegal or must be avoided, plug-ins given only their inputs and outputs by a framework that owns
+the allocator, processes whose memory pool is committed at start-up.  The test makes two calls in a row with
+different shapes, so the second one runs on an array that still holds the first call's values."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2203_17189_b200 import binding as Bd
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _case(seed, B, H, Tq, Tk, dk, causal, impl):
+    rng = np.random.default_rng(seed)
+    I = H * dk
+    bf = torch.bfloat16
+
+    def rnd(*shape, s=1.0):
+        return torch.from_numpy((rng.standard_normal(shape) * s).astype(np.float32)).to(DEV).to(bf)
+    q, k, v, do = rnd(B * Tq, I, s=0.7), rnd(B * Tk, I, s=0.7), rnd(B * Tk, I, s=0.7), rnd(B * Tq, I)
+    cq = torch.ones(B, Tq, dtype=torch.int32, device=DEV)
+    ck = torch.ones(B, Tk, dtype=torch.int32, device=DEV)
+    cq[0, Tq - 5:] = 0
+    ck[0, Tk - 7:] = 0
+    if causal:
+        ck = cq
+    bias = torch.from_numpy((rng.standard_normal((H, Tq + Tk - 1)) * 0.3).astype(np.float32)).to(DEV)
+    o = torch.empty(B * Tq, I, dtype=bf, device=DEV)
+    o32 = torch.empty(B * Tq, I, dtype=torch.float32, device=DEV)
+    lse = torch.empty(B, H, Tq, dtype=torch.float32, device=DEV)
+    Bd.t5_attention(impl, False, B, H, Tq, Tk, dk, causal, 0.25, q, k, v, o, lse, cq, ck, bias, o32=o32)
+
+    def outs():
+        return (torch.full((B * Tq, I), float("nan"), dtype=bf, device=DEV),
+                torch.full((B * Tk, I), float("nan"), dtype=bf, device=DEV),
+                torch.full((B * Tk, I), float("nan"), dtype=bf, device=DEV),
+                torch.zeros(H, Tq + Tk - 1, dtype=torch.float32, device=DEV))
+    dq0, dk0, dv0, db0 = outs()
+    delta = torch.empty(B, H, Tq, dtype=torch.float32, device=DEV)
+    Bd.t5_attention(impl, True, B, H, Tq, Tk, dk, causal, 0.25, q, k, v, o, lse, cq, ck, bias, do=do, dq=dq0,
+                    dk=dk0, dv=dv0, delta=delta, dbias_delta=db0, o32=o32)
+    dq1, dk1, dv1, db1 = outs()
+    before = torch.cuda.memory_allocated()
+    Bd.t5_attention_backward_noalloc(impl, B, H, Tq, Tk, dk, causal, 0.25, q, k, v, o, o32, lse, cq, ck, bias,
+                                     do, dq1, dk1, dv1, db1)
+    assert torch.cuda.memory_allocated() == before
+    torch.cuda.synchronize()
+    for a, b in ((dq0, dq1), (dk0, dk1), (dv0, dv1)):
+        a, b = a.float(), b.float()
+        assert torch.isfinite(b).all()
+        assert (a - b).abs().max() <= 2e-2 * a.abs().max()     # the bar the attention tests use
+    # the bias gradient is summed with atomics: same values up to summation order
+    assert (db0 - db1).abs().max() <= 1e-3 * db0.abs().max()
+
+
+@pytest.mark.parametrize("impl", [1, 0])
+def test_noalloc_backward_matches_regular_entry_point_twice(impl):
+    _case(1, 2, 3, 200, 200, 64, True, impl)
+    _case(2, 3, 2, 114, 300, 64, False, impl)      # other shape; the array still holds the first call's values
+
+
+def test_noalloc_rejects_oversized_problem():
+    t = torch.zeros(8, 64, dtype=torch.bfloat16, device=DEV)
+    f = torch.zeros(8, dtype=torch.float32, device=DEV)
+    i = torch.zeros(8, dtype=torch.int32, device=DEV)
+    with pytest.raises(Bd.T5Error) as e:
+        Bd.t5_attention_backward_noalloc(1, 4096, 32, 2048, 2048, 64, False, 1.0, t, t, t, t, f, f, i, i, None,
+                                         t, t, t, t)
+    assert e.value.code == -3
