@@ -185,6 +185,8 @@ def main():
     ap.add_argument("--workload", default="xl", choices=list(WL.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch rows")
+    ap.add_argument("--enc-layers", type=int, default=None, help="reduced depth (small profiling captures only)")
+    ap.add_argument("--dec-layers", type=int, default=None)
     ap.add_argument("--ref-rows", type=int, default=1)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--flags", type=int, default=0)
@@ -192,6 +194,10 @@ def main():
     cfg = WL.model_dims(args.workload)
     if args.batch:
         cfg["batch"] = args.batch
+    if args.enc_layers is not None:
+        cfg["n_enc_layers"] = args.enc_layers
+    if args.dec_layers is not None:
+        cfg["n_dec_layers"] = args.dec_layers
     if args.impl == "reference":
         run_reference(args, cfg)
         return
@@ -308,7 +314,7 @@ def main():
         "metric": "train_tokens_per_sec", "value": value, "unit": "tokens/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": cfg["dtype"], "data": "synthetic",
-        "config": {"workload": args.workload, "batch_rows": B, "enc_len": Te, "dec_len": Td,
+        "config": {"workload": args.workload, "layers": [cfg["n_enc_layers"], cfg["n_dec_layers"]], "batch_rows": B, "enc_len": Te, "dec_len": Td,
                    "tokens_per_step": tokens_per_step, "nonpad_tokens_per_step": nonpad,
                    "l2": f"working set {ws_bytes / 1e9:.1f} GB of activations >> 126 MB L2; no explicit flush",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
