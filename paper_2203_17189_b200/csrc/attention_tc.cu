@@ -58,6 +58,24 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
+// Common position code of n consecutive keys/queries (n = 128: one int4 per lane, n = 64: one int2),
+// or -1 if they differ.  A tile whose code equals every row's code (and lies on the allowed side of the
+// diagonal) needs no per-element mask.
+__device__ __forceinline__ int tile_code128(const int* codes, int lane) {
+  int4 c = *reinterpret_cast<const int4*>(codes + lane * 4);
+  int first = __shfl_sync(0xffffffffu, c.x, 0);
+  bool same = c.x == first && c.y == first && c.z == first && c.w == first;
+  return __all_sync(0xffffffffu, same) ? first : -1;
+}
+__device__ __forceinline__ int tile_code64(const int* codes, int lane) {
+  int2 c = *reinterpret_cast<const int2*>(codes + lane * 2);
+  int first = __shfl_sync(0xffffffffu, c.x, 0);
+  bool same = c.x == first && c.y == first;
+  return __all_sync(0xffffffffu, same) ? first : -1;
+}
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
 struct Bars {
   uint64_t ld[4];      // TMA barriers (meaning per kernel)
   uint64_t mma[2];     // MMA completion barriers
@@ -170,52 +188,62 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
       for (int c = 0; c < DK / 64; ++c)
         tma_load_3d(smem + L::kK + c * 16384, &mk, h * DK + c * 64, k0 + 128, b, bar_k);
     }
-    // pass 1: row maximum of the masked, biased scores (in log2 units)
-    float mt = -INFINITY;
-#pragma unroll 1
-    for (int c = 0; c < 4; ++c) {
+    // ---- softmax of this 128-key tile (scores in log2 units)
+    const int tcode = tile_code128(codes_s + k0, tid & 31);
+    const bool fast = tcode > 0 && __all_sync(0xffffffffu, cq == tcode) &&
+                      (!p.causal || k0 + 127 <= q0 + (warp << 5));          // warp-uniform: no mask needed
+    const float* brow = bias_s + (k0 - tid + 127);
+    const bool has_bias = p.bias_delta != nullptr;
+    constexpr bool KEEP = DK <= 64;                   // keep the 128 scores in registers between the two sweeps
+    float sc[KEEP ? 4 : 1][32];
+    auto scores = [&](int c, float (&sv)[32]) {
       uint32_t r[32];
       tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, r);
-      tmem_wait_ld();
+      tmem_wait_ld_dep(r);
+      if (has_bias) {
 #pragma unroll
-      for (int jj = 0; jj < 32; ++jj) {
-        int j = k0 + c * 32 + jj;
-        int ck = codes_s[j];
-        bool valid = ck != 0 && ck == cq && (!p.causal || j <= i);
-        float s = __uint_as_float(r[jj]) * sc2 + bias_s[j - tid + 127];
-        mt = valid ? fmaxf(mt, s) : mt;
+        for (int jj = 0; jj < 32; ++jj) sv[jj] = fmaf(__uint_as_float(r[jj]), sc2, brow[c * 32 + jj]);
+      } else {
+#pragma unroll
+        for (int jj = 0; jj < 32; ++jj) sv[jj] = __uint_as_float(r[jj]) * sc2;
       }
+      if (!fast) {
+#pragma unroll
+        for (int jj = 0; jj < 32; ++jj) {
+          int j = k0 + c * 32 + jj;
+          int ck = codes_s[j];
+          bool valid = ck != 0 && ck == cq && (!p.causal || j <= i);
+          sv[jj] = valid ? sv[jj] : -INFINITY;
+        }
+      }
+    };
+    float mt = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      float (&sv)[32] = sc[KEEP ? c : 0];
+      scores(c, sv);
+#pragma unroll
+      for (int jj = 0; jj < 32; ++jj) mt = fmaxf(mt, sv[jj]);
     }
     const float m_new = fmaxf(m_run, mt);
-    const float corr = m_run == -INFINITY ? 0.f : exp2f(m_run - m_new);
+    const float m_eff = m_new == -INFINITY ? 0.f : m_new;      // a row with no valid key so far: exp2(-inf - 0) = 0
+    const float corr = ex2_approx(m_run - m_eff);
     float lsum = 0.f;
-    // pass 2: probabilities (bf16) into the swizzled P tile
-#pragma unroll 1
-    for (int c = 0; c < 4; ++c) {
-      uint32_t r[32];
-      tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, r);
-      tmem_wait_ld();
-      float pv[32];
 #pragma unroll
-      for (int jj = 0; jj < 32; ++jj) {
-        int j = k0 + c * 32 + jj;
-        int ck = codes_s[j];
-        bool valid = ck != 0 && ck == cq && (!p.causal || j <= i);
-        float s = __uint_as_float(r[jj]) * sc2 + bias_s[j - tid + 127];
-        // the row sum uses the bf16-rounded probabilities, so the weights the MMA applies sum to one
-        float e = valid ? __bfloat162float(__float2bfloat16_rn(exp2f(s - m_new))) : 0.f;
-        pv[jj] = e;
-        lsum += e;
-      }
+    for (int c = 0; c < 4; ++c) {
+      float (&sv)[32] = sc[KEEP ? c : 0];
+      if (!KEEP) scores(c, sv);
       unsigned char* chunk = smem + L::kPo + (c >> 1) * 16384;
 #pragma unroll
       for (int q8 = 0; q8 < 4; ++q8) {
-        uint4 v;
-        v.x = pack_bf16(pv[q8 * 8 + 0], pv[q8 * 8 + 1]);
-        v.y = pack_bf16(pv[q8 * 8 + 2], pv[q8 * 8 + 3]);
-        v.z = pack_bf16(pv[q8 * 8 + 4], pv[q8 * 8 + 5]);
-        v.w = pack_bf16(pv[q8 * 8 + 6], pv[q8 * 8 + 7]);
-        store_swizzled_16B(chunk, tid, (c & 1) * 4 + q8, v);
+        uint32_t u[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          u[e] = pack_bf16(ex2_approx(sv[q8 * 8 + 2 * e] - m_eff), ex2_approx(sv[q8 * 8 + 2 * e + 1] - m_eff));
+          // the row sum uses the bf16-rounded probabilities, so the weights the MMA applies sum to one
+          lsum += bf16_lo(u[e]) + bf16_hi(u[e]);
+        }
+        store_swizzled_16B(chunk, tid, (c & 1) * 4 + q8, make_uint4(u[0], u[1], u[2], u[3]));
       }
     }
     l_run = l_run * corr + lsum;
@@ -250,9 +278,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
     for (int c = 0; c < DK / 32; ++c) {
       uint32_t r[32];
       tmem_ld_32x32b_x32(tmem_base + lane_off + 128 + c * 32, r);
-      tmem_wait_ld();
+      tmem_wait_ld_dep(r);
 #pragma unroll
-      for (int jj = 0; jj < 32; ++jj) o[c * 32 + jj] = o[c * 32 + jj] * corr + __uint_as_float(r[jj]);
+      for (int jj = 0; jj < 32; ++jj) o[c * 32 + jj] = fmaf(o[c * 32 + jj], corr, __uint_as_float(r[jj]));
     }
     tc_fence_before();
   }
@@ -301,7 +329,7 @@ struct DqLayout {
   static constexpr int kMisc = kDS + 128 * 64 * 2;
   static int bytes(int Tk) {
     int tkp = (Tk + 63) / 64 * 64;
-    return kMisc + 2 * (tkp + 128) * 4 + tkp * 4 + (int)sizeof(Bars) + 1024 + 64;
+    return kMisc + (tkp + 128) * 4 + 4 * (tkp + 32) * 4 + tkp * 4 + (int)sizeof(Bars) + 1024 + 64;
   }
 };
 
@@ -314,8 +342,11 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int tkp = (p.Tk + 63) / 64 * 64;
   float* bias_s = (float*)(smem + L::kMisc);          // [tkp + 128]
-  float* dbias_s = bias_s + tkp + 128;                // [tkp + 128]
-  int* codes_s = (int*)(dbias_s + tkp + 128);         // [tkp]
+  // bias gradient: one window per warp, indexed by (key - lane + 31); a warp's lanes touch distinct
+  // entries in one instruction, so plain read-modify-write (no atomics) is enough
+  const int wlen = tkp + 32;
+  float* dbias_s = bias_s + tkp + 128;                // [4][tkp + 32]
+  int* codes_s = (int*)(dbias_s + 4 * wlen);          // [tkp]
   Bars* bars = (Bars*)(((uintptr_t)(codes_s + tkp) + 15) & ~(uintptr_t)15);
   volatile int* abort_flag = &bars->abort_flag;
 
@@ -337,8 +368,8 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
   for (int w = tid; w < tkp + 128; w += 128) {
     int g = w - 127 - q0 + p.Tq - 1;
     bias_s[w] = (p.bias_delta && g >= 0 && g < span) ? p.bias_delta[(int64_t)h * span + g] * kLog2e : 0.f;
-    dbias_s[w] = 0.f;
   }
+  for (int w = tid; w < 4 * wlen; w += 128) dbias_s[w] = 0.f;
   for (int j = tid; j < tkp; j += 128) codes_s[j] = j < p.Tk ? p.code_k[b * p.Tk + j] : 0;
   tc_fence_before();
   __syncthreads();
@@ -409,23 +440,38 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
     ph_m ^= 1;
     if (!ok) break;
     tc_fence_after();
-#pragma unroll 1
+    const int tcode = tile_code64(codes_s + k0, tid & 31);
+    const bool fast = tcode > 0 && __all_sync(0xffffffffu, cq == tcode) &&
+                      (!p.causal || k0 + 63 <= q0 + (warp << 5));           // warp-uniform: no mask needed
+    const float* brow = bias_s + (k0 - tid + 127);
+    volatile float* dbrow = dbias_s + warp * wlen + (k0 - (tid & 31) + 31);
+    const bool has_bias = p.bias_delta != nullptr;
+#pragma unroll
     for (int c = 0; c < 2; ++c) {
       uint32_t rs[32], rp[32];
       tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, rs);
       tmem_ld_32x32b_x32(tmem_base + lane_off + 64 + c * 32, rp);
-      tmem_wait_ld();
+      tmem_wait_ld_dep(rs);
+      tmem_wait_ld_dep(rp);
       float ds[32];
 #pragma unroll
       for (int jj = 0; jj < 32; ++jj) {
-        int j = k0 + c * 32 + jj;
-        int ck = codes_s[j];
-        bool valid = ck != 0 && ck == cq && (!p.causal || j <= i) && lse2 != -INFINITY;
-        float s = __uint_as_float(rs[jj]) * sc2 + bias_s[j - tid + 127];
-        float pr = valid ? exp2f(s - lse2) : 0.f;
-        float v = pr * (__uint_as_float(rp[jj]) - dl);
-        ds[jj] = v;
-        if (want_db && valid) atomicAdd(&dbias_s[j - tid + 127], v);
+        float sv = has_bias ? fmaf(__uint_as_float(rs[jj]), sc2, brow[c * 32 + jj]) : __uint_as_float(rs[jj]) * sc2;
+        float pr = ex2_approx(sv - lse2);
+        if (!fast) {
+          int j = k0 + c * 32 + jj;
+          int ck = codes_s[j];
+          bool valid = ck != 0 && ck == cq && (!p.causal || j <= i) && lse2 != -INFINITY;
+          pr = valid ? pr : 0.f;
+        }
+        ds[jj] = pr * (__uint_as_float(rp[jj]) - dl);
+      }
+      if (want_db) {
+#pragma unroll
+        for (int jj = 0; jj < 32; ++jj) {
+          dbrow[c * 32 + jj] = dbrow[c * 32 + jj] + ds[jj];
+          __syncwarp();     // lane l+1 reads this entry in the next iteration
+        }
       }
 #pragma unroll
       for (int q8 = 0; q8 < 4; ++q8) {
@@ -479,8 +525,14 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
   tc_fence_before();
   __syncthreads();
   if (ok && want_db) {
+    // CTA-level index (key - row + 127) = warp-level index + 96 - 32 * warp
     for (int w = tid; w < tkp + 128; w += 128) {
-      float v = dbias_s[w];
+      float v = 0.f;
+#pragma unroll
+      for (int wp = 0; wp < 4; ++wp) {
+        int x = w - 96 + 32 * wp;
+        if (x >= 0 && x < wlen) v += dbias_s[wp * wlen + x];
+      }
       int g = w - 127 - q0 + p.Tq - 1;
       if (v != 0.f && g >= 0 && g < span) atomicAdd(&p.dbias_delta[(int64_t)h * span + g], v);
     }
@@ -613,23 +665,39 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
     ph_m ^= 1;
     if (!ok) break;
     tc_fence_after();
-#pragma unroll 1
+    const int tcode = tile_code64(codes_s + qb, tid & 31);
+    const bool fast = tcode > 0 && __all_sync(0xffffffffu, ck == tcode) &&
+                      (!p.causal || k0 + (warp << 5) + 31 <= qb);           // warp-uniform: no mask needed
+    const float* brow = bias_s + (tid - qb + tqp);       // element q of the tile: brow[-(q - qb)]
+    const bool has_bias = p.bias_delta != nullptr;
+#pragma unroll
     for (int c = 0; c < 2; ++c) {
       uint32_t rs[32], rp[32];
       tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, rs);
       tmem_ld_32x32b_x32(tmem_base + lane_off + 64 + c * 32, rp);
-      tmem_wait_ld();
+      tmem_wait_ld_dep(rs);
+      tmem_wait_ld_dep(rp);
       float pt[32], ds[32];
 #pragma unroll
-      for (int ii = 0; ii < 32; ++ii) {
-        int q = qb + c * 32 + ii;
-        int cq = codes_s[q];
-        float lse2 = lse_s[q];
-        bool valid = ck != 0 && ck == cq && (!p.causal || j <= q) && lse2 != -INFINITY;
-        float s = __uint_as_float(rs[ii]) * sc2 + bias_s[tid - q + tqp];
-        float pr = valid ? exp2f(s - lse2) : 0.f;
-        pt[ii] = pr;
-        ds[ii] = pr * (__uint_as_float(rp[ii]) - dl_s[q]);
+      for (int i4 = 0; i4 < 8; ++i4) {
+        const float4 l4 = *reinterpret_cast<const float4*>(lse_s + qb + c * 32 + i4 * 4);
+        const float4 d4 = *reinterpret_cast<const float4*>(dl_s + qb + c * 32 + i4 * 4);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int ii = i4 * 4 + e;
+          const float lse2 = e == 0 ? l4.x : e == 1 ? l4.y : e == 2 ? l4.z : l4.w;
+          const float dlq = e == 0 ? d4.x : e == 1 ? d4.y : e == 2 ? d4.z : d4.w;
+          float sv = has_bias ? fmaf(__uint_as_float(rs[ii]), sc2, brow[-(c * 32 + ii)]) : __uint_as_float(rs[ii]) * sc2;
+          float pr = ex2_approx(sv - lse2);
+          if (!fast) {
+            int q = qb + c * 32 + ii;
+            int cq = codes_s[q];
+            bool valid = ck != 0 && ck == cq && (!p.causal || j <= q) && lse2 != -INFINITY;
+            pr = valid ? pr : 0.f;
+          }
+          pt[ii] = pr;
+          ds[ii] = pr * (__uint_as_float(rp[ii]) - dlq);
+        }
       }
 #pragma unroll
       for (int q8 = 0; q8 < 4; ++q8) {
