@@ -84,13 +84,19 @@ struct Bars {
 };
 
 // ============================================================================ forward
+// 64-key tiles.  Tensor memory: S in columns [0,64), the output accumulator O in [64, 64+DK).
+// Per tile one wait: thread 0 issues PV(t) and right behind it S(t+1) with a single commit, so the
+// softmax of tile t+1 starts as soon as both are done.  O stays in tensor memory and is rescaled in
+// place (tcgen05.ld / st) only when a row maximum of the warp changed; this keeps the register count
+// low enough for four CTAs per SM, which is what hides the MMA and TMA latencies.
 template <int DK>
 struct FwdLayout {
-  static constexpr int kTile = 128 * DK * 2;          // Q, K or V tile bytes
-  static constexpr int kP = 128 * 128 * 2;
-  static constexpr int kQ = 0, kK = kTile, kV = 2 * kTile, kPo = 3 * kTile, kMisc = 3 * kTile + kP;
+  static constexpr int kQBytes = 128 * DK * 2;
+  static constexpr int kKVBytes = 64 * DK * 2;          // one K or V tile
+  static constexpr int kP = 128 * 64 * 2;
+  static constexpr int kQ = 0, kK = kQBytes, kV = kK + kKVBytes, kPo = kV + kKVBytes, kMisc = kPo + kP;
   static int bytes(int Tk) {
-    int tkp = (Tk + 127) / 128 * 128;
+    int tkp = (Tk + 63) / 64 * 64;
     return kMisc + (tkp + 128) * 4 + tkp * 4 + (int)sizeof(Bars) + 1024 + 64;
   }
 };
@@ -102,17 +108,17 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
   using L = FwdLayout<DK>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  const int tkp = (p.Tk + 127) / 128 * 128;
-  float* bias_s = (float*)(smem + L::kMisc);          // [tkp + 128]
+  const int tkp = (p.Tk + 63) / 64 * 64;
+  float* bias_s = (float*)(smem + L::kMisc);          // [tkp + 128], entry (key - row + 127), log2 units
   int* codes_s = (int*)(bias_s + tkp + 128);          // [tkp]
   Bars* bars = (Bars*)(((uintptr_t)(codes_s + tkp) + 15) & ~(uintptr_t)15);
   volatile int* abort_flag = &bars->abort_flag;
 
   const int tid = threadIdx.x, warp = tid >> 5;
   const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * 128;
-  int n_kt = (p.Tk + 127) / 128;
-  if (p.causal) n_kt = min(n_kt, (q0 + 127) / 128 + 1);
-  constexpr uint32_t kTmemCols = 256;
+  int n_kt = (p.Tk + 63) / 64;
+  if (p.causal) n_kt = min(n_kt, (q0 + 127) / 64 + 1);
+  constexpr uint32_t kTmemCols = DK == 64 ? 128 : 256;
 
   if (tid == 0) {
     for (int i = 0; i < 4; ++i) mbar_init(&bars->ld[i], 1);
@@ -136,175 +142,184 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
   uint64_t* bar_k = &bars->ld[0];
   uint64_t* bar_v = &bars->ld[1];
   uint64_t* bar_m = &bars->mma[0];
+  constexpr uint32_t idesc_s = make_idesc(128, 64, false, false);
+  constexpr uint32_t idesc_pv = make_idesc(128, DK, false, true);
+  uint32_t ph_k = 0, ph_v = 0, ph_m = 0;
+  bool ok = true, pend_k = false, pend_v = false;      // pend_*: a load of that tile is in flight (thread 0 only)
+
+  auto load_k = [&](int t) {
+    pend_k = true;
+    mbar_arrive_expect_tx(bar_k, L::kKVBytes);
+#pragma unroll
+    for (int c = 0; c < DK / 64; ++c) tma_load_3d(smem + L::kK + c * 8192, &mk, h * DK + c * 64, t * 64, b, bar_k);
+  };
+  auto load_v = [&](int t) {
+    pend_v = true;
+    mbar_arrive_expect_tx(bar_v, L::kKVBytes);
+#pragma unroll
+    for (int c = 0; c < DK / 64; ++c) tma_load_3d(smem + L::kV + c * 8192, &mv, h * DK + c * 64, t * 64, b, bar_v);
+  };
+  auto issue_s = [&]() {      // S = Q K^T of the tile in the K buffer; returns false if its load never arrived
+    if (!mbar_wait(bar_k, ph_k, abort_flag, p.status, 11)) return false;
+    ph_k ^= 1;
+    pend_k = false;
+    tc_fence_after();
+#pragma unroll
+    for (int kk = 0; kk < DK / 16; ++kk)
+      umma_bf16(tmem_base, desc_k(sQ + (kk >> 2) * 16384 + (kk & 3) * 32), desc_k(sK + (kk >> 2) * 8192 + (kk & 3) * 32),
+                idesc_s, kk != 0);
+    return true;
+  };
 
   if (tid == 0) {
-    mbar_arrive_expect_tx(bar_k, 2 * L::kTile);
+    pend_k = true;
+    mbar_arrive_expect_tx(bar_k, L::kQBytes + L::kKVBytes);
 #pragma unroll
     for (int c = 0; c < DK / 64; ++c) {
       tma_load_3d(smem + L::kQ + c * 16384, &mq, h * DK + c * 64, q0, b, bar_k);
-      tma_load_3d(smem + L::kK + c * 16384, &mk, h * DK + c * 64, 0, b, bar_k);
+      tma_load_3d(smem + L::kK + c * 8192, &mk, h * DK + c * 64, 0, b, bar_k);
     }
-    mbar_arrive_expect_tx(bar_v, L::kTile);
-#pragma unroll
-    for (int c = 0; c < DK / 64; ++c) tma_load_3d(smem + L::kV + c * 16384, &mv, h * DK + c * 64, 0, b, bar_v);
+    load_v(0);
+    if (issue_s()) umma_commit(bar_m);
   }
 
   const int i = q0 + tid;
   const int cq = i < p.Tq ? p.code_q[b * p.Tq + i] : 0;
   float m_run = -INFINITY, l_run = 0.f;
-  float o[DK];
-#pragma unroll
-  for (int d = 0; d < DK; ++d) o[d] = 0.f;
   const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
   const float sc2 = p.scale * kLog2e;
-  uint32_t ph_k = 0, ph_v = 0, ph_m = 0;
-  bool ok = true, pend_k = true, pend_v = true;      // pend_*: a load of that tile is in flight (thread 0 only)
-  constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
-  constexpr uint32_t idesc_pv = make_idesc(128, DK, false, true);
+  const bool has_bias = p.bias_delta != nullptr;
 
   for (int t = 0; t < n_kt && ok; ++t) {
-    const int k0 = t * 128;
-    if (tid == 0) {
-      if (mbar_wait(bar_k, ph_k, abort_flag, p.status, 11)) {
-        ph_k ^= 1;
-        pend_k = false;
-        tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < DK / 16; ++kk) {
-          uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
-          umma_bf16(tmem_base, desc_k(sQ + off), desc_k(sK + off), idesc_s, kk != 0);
-        }
-        umma_commit(bar_m);
-      }
-    }
-    ok = mbar_wait(bar_m, ph_m, abort_flag, p.status, 12);
+    const int k0 = t * 64;
+    ok = mbar_wait(bar_m, ph_m, abort_flag, p.status, 12);      // S(t) ready, PV(t-1) done
     ph_m ^= 1;
     if (!ok) break;
     tc_fence_after();
-    if (tid == 0 && t + 1 < n_kt) {     // K tile is free again: fetch the next one
-      pend_k = true;
-      mbar_arrive_expect_tx(bar_k, L::kTile);
-#pragma unroll
-      for (int c = 0; c < DK / 64; ++c)
-        tma_load_3d(smem + L::kK + c * 16384, &mk, h * DK + c * 64, k0 + 128, b, bar_k);
+    if (tid == 0) {
+      if (t + 1 < n_kt) load_k(t + 1);       // K buffer: S(t) has consumed it
+      if (t > 0) load_v(t);                  // V buffer: PV(t-1) has consumed it
     }
-    // ---- softmax of this 128-key tile (scores in log2 units)
-    const int tcode = tile_code128(codes_s + k0, tid & 31);
+    // ---- softmax of this 64-key tile (scores in log2 units)
+    const int tcode = tile_code64(codes_s + k0, tid & 31);
     const bool fast = tcode > 0 && __all_sync(0xffffffffu, cq == tcode) &&
-                      (!p.causal || k0 + 127 <= q0 + (warp << 5));          // warp-uniform: no mask needed
+                      (!p.causal || k0 + 63 <= q0 + (warp << 5));          // warp-uniform: no mask needed
     const float* brow = bias_s + (k0 - tid + 127);
-    const bool has_bias = p.bias_delta != nullptr;
-    constexpr bool KEEP = DK <= 64;                   // keep the 128 scores in registers between the two sweeps
-    float sc[KEEP ? 4 : 1][32];
-    auto scores = [&](int c, float (&sv)[32]) {
-      uint32_t r[32];
-      tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, r);
-      tmem_wait_ld_dep(r);
-      if (has_bias) {
+    float sc[2][32];
+    {
+      uint32_t r[2][32];
+      tmem_ld_32x32b_x32(tmem_base + lane_off, r[0]);
+      tmem_ld_32x32b_x32(tmem_base + lane_off + 32, r[1]);
 #pragma unroll
-        for (int jj = 0; jj < 32; ++jj) sv[jj] = fmaf(__uint_as_float(r[jj]), sc2, brow[c * 32 + jj]);
-      } else {
+      for (int c = 0; c < 2; ++c) {
+        tmem_wait_ld_dep(r[c]);
+        if (has_bias) {
 #pragma unroll
-        for (int jj = 0; jj < 32; ++jj) sv[jj] = __uint_as_float(r[jj]) * sc2;
-      }
-      if (!fast) {
+          for (int jj = 0; jj < 32; ++jj) sc[c][jj] = fmaf(__uint_as_float(r[c][jj]), sc2, brow[c * 32 + jj]);
+        } else {
 #pragma unroll
-        for (int jj = 0; jj < 32; ++jj) {
-          int j = k0 + c * 32 + jj;
-          int ck = codes_s[j];
-          bool valid = ck != 0 && ck == cq && (!p.causal || j <= i);
-          sv[jj] = valid ? sv[jj] : -INFINITY;
+          for (int jj = 0; jj < 32; ++jj) sc[c][jj] = __uint_as_float(r[c][jj]) * sc2;
+        }
+        if (!fast) {
+#pragma unroll
+          for (int jj = 0; jj < 32; ++jj) {
+            int j = k0 + c * 32 + jj;
+            int ck = codes_s[j];
+            bool valid = ck != 0 && ck == cq && (!p.causal || j <= i);
+            sc[c][jj] = valid ? sc[c][jj] : -INFINITY;
+          }
         }
       }
-    };
-    float mt = -INFINITY;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      float (&sv)[32] = sc[KEEP ? c : 0];
-      scores(c, sv);
-#pragma unroll
-      for (int jj = 0; jj < 32; ++jj) mt = fmaxf(mt, sv[jj]);
     }
-    const float m_new = fmaxf(m_run, mt);
+    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+    for (int c = 0; c < 2; ++c)
+#pragma unroll
+      for (int jj = 0; jj < 32; jj += 4) {
+        mx[0] = fmaxf(mx[0], sc[c][jj]); mx[1] = fmaxf(mx[1], sc[c][jj + 1]);
+        mx[2] = fmaxf(mx[2], sc[c][jj + 2]); mx[3] = fmaxf(mx[3], sc[c][jj + 3]);
+      }
+    const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])));
     const float m_eff = m_new == -INFINITY ? 0.f : m_new;      // a row with no valid key so far: exp2(-inf - 0) = 0
     const float corr = ex2_approx(m_run - m_eff);
-    float lsum = 0.f;
+    // rescale the accumulator rows of this warp if any of their maxima moved
+    if (t > 0 && __any_sync(0xffffffffu, m_new != m_run)) {
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      float (&sv)[32] = sc[KEEP ? c : 0];
-      if (!KEEP) scores(c, sv);
-      unsigned char* chunk = smem + L::kPo + (c >> 1) * 16384;
+      for (int c = 0; c < DK / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(tmem_base + lane_off + 64 + c * 32, r);
+        tmem_wait_ld_dep(r);
+#pragma unroll
+        for (int jj = 0; jj < 32; ++jj) r[jj] = __float_as_uint(__uint_as_float(r[jj]) * corr);
+        tmem_st_32x32b_x32(tmem_base + lane_off + 64 + c * 32, r);
+      }
+      tmem_wait_st();
+    }
+    float ls[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < 2; ++c)
 #pragma unroll
       for (int q8 = 0; q8 < 4; ++q8) {
         uint32_t u[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          u[e] = pack_bf16(ex2_approx(sv[q8 * 8 + 2 * e] - m_eff), ex2_approx(sv[q8 * 8 + 2 * e + 1] - m_eff));
+          u[e] = pack_bf16(ex2_approx(sc[c][q8 * 8 + 2 * e] - m_eff), ex2_approx(sc[c][q8 * 8 + 2 * e + 1] - m_eff));
           // the row sum uses the bf16-rounded probabilities, so the weights the MMA applies sum to one
-          lsum += bf16_lo(u[e]) + bf16_hi(u[e]);
+          ls[e] += bf16_lo(u[e]) + bf16_hi(u[e]);
         }
-        store_swizzled_16B(chunk, tid, (c & 1) * 4 + q8, make_uint4(u[0], u[1], u[2], u[3]));
+        store_swizzled_16B(smem + L::kPo, tid, c * 4 + q8, make_uint4(u[0], u[1], u[2], u[3]));
       }
-    }
-    l_run = l_run * corr + lsum;
+    l_run = l_run * corr + ((ls[0] + ls[1]) + (ls[2] + ls[3]));
     m_run = m_new;
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
     if (tid == 0) {
-      if (mbar_wait(bar_v, ph_v, abort_flag, p.status, 13)) {
+      bool good = mbar_wait(bar_v, ph_v, abort_flag, p.status, 13);
+      if (good) {
         ph_v ^= 1;
         pend_v = false;
         tc_fence_after();
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          umma_bf16(tmem_base + 128, desc_k(sP + (ks >> 2) * 16384 + (ks & 3) * 32), desc_mn(sV + ks * 2048, 16384),
-                    idesc_pv, ks != 0);
-        umma_commit(bar_m);
+        for (int ks = 0; ks < 4; ++ks)
+          umma_bf16(tmem_base + 64, desc_k(sP + ks * 32), desc_mn(sV + ks * 2048, 8192), idesc_pv, (t | ks) != 0);
+        if (t + 1 < n_kt) good = issue_s();
+        if (good) umma_commit(bar_m);
       }
     }
-    ok = mbar_wait(bar_m, ph_m, abort_flag, p.status, 14);
-    ph_m ^= 1;
-    if (!ok) break;
+  }
+  if (ok) ok = mbar_wait(bar_m, ph_m, abort_flag, p.status, 14);   // last PV done
+  if (ok) {
     tc_fence_after();
-    if (tid == 0 && t + 1 < n_kt) {
-      pend_v = true;
-      mbar_arrive_expect_tx(bar_v, L::kTile);
-#pragma unroll
-      for (int c = 0; c < DK / 64; ++c)
-        tma_load_3d(smem + L::kV + c * 16384, &mv, h * DK + c * 64, k0 + 128, b, bar_v);
-    }
+    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+    bf16* orow = (bf16*)p.out0 + (int64_t)(b * p.Tq + i) * p.ld0 + h * DK;
+    float* o32 = p.o32 ? p.o32 + (int64_t)(b * p.Tq + i) * p.ldo32 + h * DK : nullptr;
 #pragma unroll
     for (int c = 0; c < DK / 32; ++c) {
       uint32_t r[32];
-      tmem_ld_32x32b_x32(tmem_base + lane_off + 128 + c * 32, r);
+      tmem_ld_32x32b_x32(tmem_base + lane_off + 64 + c * 32, r);
       tmem_wait_ld_dep(r);
+      if (i < p.Tq) {
 #pragma unroll
-      for (int jj = 0; jj < 32; ++jj) o[c * 32 + jj] = fmaf(o[c * 32 + jj], corr, __uint_as_float(r[jj]));
-    }
-    tc_fence_before();
-  }
-
-  if (ok && i < p.Tq) {
-    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-    bf16* orow = (bf16*)p.out0 + (int64_t)(b * p.Tq + i) * p.ld0 + h * DK;
+        for (int d = 0; d < 32; d += 8) {
+          uint4 v;
+          v.x = pack_bf16(__uint_as_float(r[d]) * inv, __uint_as_float(r[d + 1]) * inv);
+          v.y = pack_bf16(__uint_as_float(r[d + 2]) * inv, __uint_as_float(r[d + 3]) * inv);
+          v.z = pack_bf16(__uint_as_float(r[d + 4]) * inv, __uint_as_float(r[d + 5]) * inv);
+          v.w = pack_bf16(__uint_as_float(r[d + 6]) * inv, __uint_as_float(r[d + 7]) * inv);
+          *reinterpret_cast<uint4*>(orow + c * 32 + d) = v;
+        }
+        if (o32) {
 #pragma unroll
-    for (int d = 0; d < DK; d += 8) {
-      uint4 v;
-      v.x = pack_bf16(o[d] * inv, o[d + 1] * inv);
-      v.y = pack_bf16(o[d + 2] * inv, o[d + 3] * inv);
-      v.z = pack_bf16(o[d + 4] * inv, o[d + 5] * inv);
-      v.w = pack_bf16(o[d + 6] * inv, o[d + 7] * inv);
-      *reinterpret_cast<uint4*>(orow + d) = v;
+          for (int d = 0; d < 32; d += 4)
+            *reinterpret_cast<float4*>(o32 + c * 32 + d) =
+                make_float4(__uint_as_float(r[d]) * inv, __uint_as_float(r[d + 1]) * inv,
+                            __uint_as_float(r[d + 2]) * inv, __uint_as_float(r[d + 3]) * inv);
+        }
+      }
     }
-    if (p.o32) {
-      float* o32 = p.o32 + (int64_t)(b * p.Tq + i) * p.ldo32 + h * DK;
-#pragma unroll
-      for (int d = 0; d < DK; d += 4)
-        *reinterpret_cast<float4*>(o32 + d) = make_float4(o[d] * inv, o[d + 1] * inv, o[d + 2] * inv, o[d + 3] * inv);
-    }
-    // natural-log log-sum-exp of the (unscaled-by-log2e) scores
-    p.lse[(int64_t)(b * p.H + h) * p.Tq + i] = l_run > 0.f ? (m_run + log2f(l_run)) / kLog2e : -INFINITY;
+    // natural-log log-sum-exp of the scores
+    if (i < p.Tq) p.lse[(int64_t)(b * p.H + h) * p.Tq + i] = l_run > 0.f ? (m_run + log2f(l_run)) / kLog2e : -INFINITY;
   }
   if (!ok && tid == 0) {   // let TMA loads that are still in flight land before the CTA exits
     long long t0 = clock64();
@@ -444,19 +459,23 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
     const bool fast = tcode > 0 && __all_sync(0xffffffffu, cq == tcode) &&
                       (!p.causal || k0 + 63 <= q0 + (warp << 5));           // warp-uniform: no mask needed
     const float* brow = bias_s + (k0 - tid + 127);
-    volatile float* dbrow = dbias_s + warp * wlen + (k0 - (tid & 31) + 31);
+    const int lane = tid & 31;
+    float* dbwin = dbias_s + warp * wlen + k0;        // this warp's window; entry = key - (row in warp) + 31
     const bool has_bias = p.bias_delta != nullptr;
+    uint32_t rs[2][32], rp[2][32];
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
-      uint32_t rs[32], rp[32];
-      tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, rs);
-      tmem_ld_32x32b_x32(tmem_base + lane_off + 64 + c * 32, rp);
-      tmem_wait_ld_dep(rs);
-      tmem_wait_ld_dep(rp);
+      tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, rs[c]);
+      tmem_ld_32x32b_x32(tmem_base + lane_off + 64 + c * 32, rp[c]);
+    }
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      tmem_wait_ld_dep(rs[c]);
+      tmem_wait_ld_dep(rp[c]);
       float ds[32];
 #pragma unroll
       for (int jj = 0; jj < 32; ++jj) {
-        float sv = has_bias ? fmaf(__uint_as_float(rs[jj]), sc2, brow[c * 32 + jj]) : __uint_as_float(rs[jj]) * sc2;
+        float sv = has_bias ? fmaf(__uint_as_float(rs[c][jj]), sc2, brow[c * 32 + jj]) : __uint_as_float(rs[c][jj]) * sc2;
         float pr = ex2_approx(sv - lse2);
         if (!fast) {
           int j = k0 + c * 32 + jj;
@@ -464,14 +483,22 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
           bool valid = ck != 0 && ck == cq && (!p.causal || j <= i) && lse2 != -INFINITY;
           pr = valid ? pr : 0.f;
         }
-        ds[jj] = pr * (__uint_as_float(rp[jj]) - dl);
+        ds[jj] = pr * (__uint_as_float(rp[c][jj]) - dl);
       }
       if (want_db) {
+        // Diagonal sums of this warp's 32 x 32 block without atomics: at step t lane l takes column t of
+        // row (l + t) mod 32, which lies on diagonal (col - row) = -l when l + t < 32 and 32 - l otherwise.
+        float a0 = 0.f, a1 = 0.f;
 #pragma unroll
-        for (int jj = 0; jj < 32; ++jj) {
-          dbrow[c * 32 + jj] = dbrow[c * 32 + jj] + ds[jj];
-          __syncwarp();     // lane l+1 reads this entry in the next iteration
+        for (int t = 0; t < 32; ++t) {
+          float v = __shfl_sync(0xffffffffu, ds[t], (lane + t) & 31);
+          if (lane + t < 32) a0 += v; else a1 += v;
         }
+        // window entry (col - row + 31): diagonal -l -> 31 - l, diagonal 32 - l -> 63 - l; distinct per lane
+        dbwin[c * 32 + 31 - lane] += a0;
+        __syncwarp();
+        dbwin[c * 32 + 63 - lane] += a1;
+        __syncwarp();
       }
 #pragma unroll
       for (int q8 = 0; q8 < 4; ++q8) {
@@ -670,11 +697,16 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
                       (!p.causal || k0 + (warp << 5) + 31 <= qb);           // warp-uniform: no mask needed
     const float* brow = bias_s + (tid - qb + tqp);       // element q of the tile: brow[-(q - qb)]
     const bool has_bias = p.bias_delta != nullptr;
+    uint32_t rsa[2][32], rpa[2][32];
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
-      uint32_t rs[32], rp[32];
-      tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, rs);
-      tmem_ld_32x32b_x32(tmem_base + lane_off + 64 + c * 32, rp);
+      tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, rsa[c]);
+      tmem_ld_32x32b_x32(tmem_base + lane_off + 64 + c * 32, rpa[c]);
+    }
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      uint32_t (&rs)[32] = rsa[c];
+      uint32_t (&rp)[32] = rpa[c];
       tmem_wait_ld_dep(rs);
       tmem_wait_ld_dep(rp);
       float pt[32], ds[32];
@@ -832,8 +864,8 @@ template <int DK>
 cudaError_t fwd_launch(const AttnArgs& a, int* status, cudaStream_t st) {
   CUtensorMap mq, mk, mv;
   int I = a.H * DK;
-  if (!make_map3(&mq, a.Q, I, a.Tq, a.B, a.ldq, 128) || !make_map3(&mk, a.K, I, a.Tk, a.B, a.ldk, 128) ||
-      !make_map3(&mv, a.V, I, a.Tk, a.B, a.ldv, 128))
+  if (!make_map3(&mq, a.Q, I, a.Tq, a.B, a.ldq, 128) || !make_map3(&mk, a.K, I, a.Tk, a.B, a.ldk, 64) ||
+      !make_map3(&mv, a.V, I, a.Tk, a.B, a.ldv, 64))
     return cudaErrorInvalidValue;
   int smem = FwdLayout<DK>::bytes(a.Tk);
   cudaError_t e = cudaFuncSetAttribute(attn_fwd_tc_kernel<DK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
