@@ -22,9 +22,12 @@
 
 #include <math.h>
 
+#include <algorithm>
+
 namespace {
 
 using namespace tc;
+using std::max;
 
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -340,7 +343,7 @@ struct DqLayout {
   static constexpr int kQ = 0, kDO = 128 * DK * 2, kKV0 = 2 * 128 * DK * 2;
   static constexpr int kKVTile = 64 * DK * 2;                   // one K or V tile (64 keys)
   static constexpr int kStage = 2 * kKVTile;                    // K then V
-  static constexpr int kDS = kKV0 + 2 * kStage;                 // [128 x 64] bf16
+  static constexpr int kDS = kKV0 + 3 * kStage;                 // [128 x 64] bf16
   static constexpr int kMisc = kDS + 128 * 64 * 2;
   static int bytes(int Tk) {
     int tkp = (Tk + 63) / 64 * 64;
@@ -378,6 +381,29 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
     bars->abort_flag = 0;
     fence_barrier_init();
   }
+  uint64_t* bar_q = &bars->ld[0];        // Q and dO
+  uint64_t* bar_kv = &bars->ld[1];       // [3] stages: ld[1..3]
+  uint64_t* bar_m = &bars->mma[0];       // S(t), dP(t) ready and dQ(t-1) done
+  auto load_kv = [&](int t) {
+    int st = t % 3;
+    unsigned char* base = smem + L::kKV0 + st * L::kStage;
+    mbar_arrive_expect_tx(&bar_kv[st], L::kStage);
+#pragma unroll
+    for (int c = 0; c < DK / 64; ++c) {
+      tma_load_3d(base + c * 8192, &mk, h * DK + c * 64, t * 64, b, &bar_kv[st]);
+      tma_load_3d(base + L::kKVTile + c * 8192, &mv, h * DK + c * 64, t * 64, b, &bar_kv[st]);
+    }
+  };
+  if (tid == 0) {      // loads go out before the rest of the set-up so that their latency overlaps it
+    mbar_arrive_expect_tx(bar_q, 2 * 128 * DK * 2);
+#pragma unroll
+    for (int c = 0; c < DK / 64; ++c) {
+      tma_load_3d(smem + L::kQ + c * 16384, &mq, h * DK + c * 64, q0, b, bar_q);
+      tma_load_3d(smem + L::kDO + c * 16384, &mdo, h * DK + c * 64, q0, b, bar_q);
+    }
+    load_kv(0);
+    if (n_kt > 1) load_kv(1);
+  }
   if (warp == 0) tmem_alloc(&bars->tmem, kTmemCols);
   const int span = p.Tq + p.Tk - 1;
   for (int w = tid; w < tkp + 128; w += 128) {
@@ -391,30 +417,6 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem;
   const uint32_t sQ = smem_u32(smem + L::kQ), sDO = smem_u32(smem + L::kDO), sDS = smem_u32(smem + L::kDS);
-  uint64_t* bar_q = &bars->ld[0];        // Q and dO
-  uint64_t* bar_kv = &bars->ld[1];       // [2] stages: ld[1], ld[2]
-  uint64_t* bar_m = &bars->mma[0];       // S and dP ready
-  uint64_t* bar_dq = &bars->mma[1];      // dQ MMA of the tile done
-
-  auto load_kv = [&](int t) {
-    int st = t & 1;
-    unsigned char* base = smem + L::kKV0 + st * L::kStage;
-    mbar_arrive_expect_tx(&bar_kv[st], L::kStage);
-#pragma unroll
-    for (int c = 0; c < DK / 64; ++c) {
-      tma_load_3d(base + c * 8192, &mk, h * DK + c * 64, t * 64, b, &bar_kv[st]);
-      tma_load_3d(base + L::kKVTile + c * 8192, &mv, h * DK + c * 64, t * 64, b, &bar_kv[st]);
-    }
-  };
-  if (tid == 0) {
-    mbar_arrive_expect_tx(bar_q, 2 * 128 * DK * 2);
-#pragma unroll
-    for (int c = 0; c < DK / 64; ++c) {
-      tma_load_3d(smem + L::kQ + c * 16384, &mq, h * DK + c * 64, q0, b, bar_q);
-      tma_load_3d(smem + L::kDO + c * 16384, &mdo, h * DK + c * 64, q0, b, bar_q);
-    }
-    load_kv(0);
-  }
 
   const int i = q0 + tid;
   const bool row_in = i < p.Tq;
@@ -423,38 +425,42 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
   const float dl = row_in ? p.delta[(int64_t)(b * p.H + h) * p.Tq + i] : 0.f;
   const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
   const float sc2 = p.scale * kLog2e;
-  uint32_t ph_kv[2] = {0, 0}, ph_m = 0, ph_dq = 0;
+  uint32_t ph_kv[3] = {0, 0, 0}, ph_m = 0;
   bool ok = true;
   constexpr uint32_t idesc_s = make_idesc(128, 64, false, false);
   constexpr uint32_t idesc_dq = make_idesc(128, DK, false, true);
 
-  if (tid == 0) ok = mbar_wait(bar_q, 0, abort_flag, p.status, 21);
+  // S = Q K^T and dP = dO V^T of tile t (thread 0); false if the tile's load never arrived
+  auto issue_s_dp = [&](int t) {
+    const int st = t % 3;
+    if (!mbar_wait(&bar_kv[st], ph_kv[st], abort_flag, p.status, 22)) return false;
+    ph_kv[st] ^= 1;
+    tc_fence_after();
+    const uint32_t sK = smem_u32(smem + L::kKV0 + st * L::kStage), sV = sK + L::kKVTile;
+#pragma unroll
+    for (int kk = 0; kk < DK / 16; ++kk) {
+      uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
+      umma_bf16(tmem_base, desc_k(sQ + oa), desc_k(sK + ob), idesc_s, kk != 0);
+    }
+#pragma unroll
+    for (int kk = 0; kk < DK / 16; ++kk) {
+      uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
+      umma_bf16(tmem_base + 64, desc_k(sDO + oa), desc_k(sV + ob), idesc_s, kk != 0);
+    }
+    return true;
+  };
+  if (tid == 0) {
+    ok = mbar_wait(bar_q, 0, abort_flag, p.status, 21);
+    if (ok && issue_s_dp(0)) umma_commit(bar_m);
+  }
 
   for (int t = 0; t < n_kt && ok; ++t) {
-    const int k0 = t * 64, st = t & 1;
-    const uint32_t sK = smem_u32(smem + L::kKV0 + st * L::kStage), sV = sK + L::kKVTile;
-    if (tid == 0) {
-      if (t + 1 < n_kt) load_kv(t + 1);      // the other stage was released by the dQ wait of tile t-1
-      if (mbar_wait(&bar_kv[st], ph_kv[st], abort_flag, p.status, 22)) {
-        tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < DK / 16; ++kk) {
-          uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
-          umma_bf16(tmem_base, desc_k(sQ + oa), desc_k(sK + ob), idesc_s, kk != 0);
-        }
-#pragma unroll
-        for (int kk = 0; kk < DK / 16; ++kk) {
-          uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
-          umma_bf16(tmem_base + 64, desc_k(sDO + oa), desc_k(sV + ob), idesc_s, kk != 0);
-        }
-        umma_commit(bar_m);
-      }
-    }
-    ph_kv[st] ^= 1;
+    const int k0 = t * 64;
     ok = mbar_wait(bar_m, ph_m, abort_flag, p.status, 23);
     ph_m ^= 1;
     if (!ok) break;
     tc_fence_after();
+    if (tid == 0 && t + 2 < n_kt) load_kv(t + 2);      // its stage held tile t-1, whose MMAs are all done
     const int tcode = tile_code64(codes_s + k0, tid & 31);
     const bool fast = tcode > 0 && __all_sync(0xffffffffu, cq == tcode) &&
                       (!p.causal || k0 + 63 <= q0 + (warp << 5));           // warp-uniform: no mask needed
@@ -515,14 +521,16 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
     __syncthreads();
     if (tid == 0) {
       tc_fence_after();
+      const uint32_t sK = smem_u32(smem + L::kKV0 + (t % 3) * L::kStage);
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks)
         umma_bf16(tmem_base + 128, desc_k(sDS + ks * 32), desc_mn(sK + ks * 2048, 8192), idesc_dq, (t | ks) != 0);
-      umma_commit(bar_dq);
+      bool good = true;
+      if (t + 1 < n_kt) good = issue_s_dp(t + 1);      // the scores of tile t are in registers by now
+      if (good) umma_commit(bar_m);
     }
-    ok = mbar_wait(bar_dq, ph_dq, abort_flag, p.status, 24);   // dS tile and this K/V stage are free again
-    ph_dq ^= 1;
   }
+  if (ok) ok = mbar_wait(bar_m, ph_m, abort_flag, p.status, 24);   // last dQ MMA done
 
   if (ok) {
     tc_fence_after();
@@ -612,6 +620,29 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
     bars->abort_flag = 0;
     fence_barrier_init();
   }
+  uint64_t* bar_kv = &bars->ld[0];
+  uint64_t* bar_qd = &bars->ld[1];       // [2] stages
+  uint64_t* bar_m = &bars->mma[0];       // S^T(t), dP^T(t) ready and the accumulating MMAs of tile t-1 done
+  auto load_qd = [&](int t) {
+    int st = t & 1;
+    unsigned char* base = smem + L::kQD0 + st * L::kStage;
+    mbar_arrive_expect_tx(&bar_qd[st], L::kStage);
+#pragma unroll
+    for (int c = 0; c < DK / 64; ++c) {
+      tma_load_3d(base + c * 8192, &mq, h * DK + c * 64, t * 64, b, &bar_qd[st]);
+      tma_load_3d(base + L::kQTile + c * 8192, &mdo, h * DK + c * 64, t * 64, b, &bar_qd[st]);
+    }
+  };
+  if (tid == 0 && t_begin < n_qt) {      // loads go out before the rest of the set-up so that their latency overlaps it
+    mbar_arrive_expect_tx(bar_kv, 2 * 128 * DK * 2);
+#pragma unroll
+    for (int c = 0; c < DK / 64; ++c) {
+      tma_load_3d(smem + L::kK + c * 16384, &mk, h * DK + c * 64, k0, b, bar_kv);
+      tma_load_3d(smem + L::kV + c * 16384, &mv, h * DK + c * 64, k0, b, bar_kv);
+    }
+    load_qd(t_begin);
+    if (t_begin + 1 < n_qt) load_qd(t_begin + 1);
+  }
   if (warp == 0) tmem_alloc(&bars->tmem, kTmemCols);
   const int span = p.Tq + p.Tk - 1;
   // distance of (key j = k0 + tid, query i): j - i ; window index w = tid - i + tqp  in [1, tqp + 127]
@@ -631,67 +662,48 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
   const uint32_t tmem_base = bars->tmem;
   const uint32_t sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV), sPt = smem_u32(smem + L::kPt),
                  sDSt = smem_u32(smem + L::kDSt);
-  uint64_t* bar_kv = &bars->ld[0];
-  uint64_t* bar_qd = &bars->ld[1];       // [2] stages
-  uint64_t* bar_m = &bars->mma[0];
-  uint64_t* bar_acc = &bars->mma[1];
-
-  auto load_qd = [&](int t) {
-    int st = t & 1;
-    unsigned char* base = smem + L::kQD0 + st * L::kStage;
-    mbar_arrive_expect_tx(&bar_qd[st], L::kStage);
-#pragma unroll
-    for (int c = 0; c < DK / 64; ++c) {
-      tma_load_3d(base + c * 8192, &mq, h * DK + c * 64, t * 64, b, &bar_qd[st]);
-      tma_load_3d(base + L::kQTile + c * 8192, &mdo, h * DK + c * 64, t * 64, b, &bar_qd[st]);
-    }
-  };
-  if (tid == 0 && t_begin < n_qt) {
-    mbar_arrive_expect_tx(bar_kv, 2 * 128 * DK * 2);
-#pragma unroll
-    for (int c = 0; c < DK / 64; ++c) {
-      tma_load_3d(smem + L::kK + c * 16384, &mk, h * DK + c * 64, k0, b, bar_kv);
-      tma_load_3d(smem + L::kV + c * 16384, &mv, h * DK + c * 64, k0, b, bar_kv);
-    }
-    load_qd(t_begin);
-  }
-
   const int j = k0 + tid;
   const bool row_in = j < p.Tk;
   const int ck = row_in ? p.code_k[b * p.Tk + j] : 0;
   const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
   const float sc2 = p.scale * kLog2e;
-  uint32_t ph_qd[2] = {0, 0}, ph_m = 0, ph_acc = 0;
+  uint32_t ph_qd[2] = {0, 0}, ph_m = 0;
   bool ok = true;
   constexpr uint32_t idesc_s = make_idesc(128, 64, false, false);
   constexpr uint32_t idesc_acc = make_idesc(128, DK, false, true);
-  if (tid == 0 && t_begin < n_qt) ok = mbar_wait(bar_kv, 0, abort_flag, p.status, 31);
+  // S^T = K Q^T and dP^T = V dO^T of query tile t (thread 0); false if the tile's load never arrived
+  auto issue_st = [&](int t) {
+    const int st = t & 1;
+    if (!mbar_wait(&bar_qd[st], ph_qd[st], abort_flag, p.status, 32)) return false;
+    ph_qd[st] ^= 1;
+    tc_fence_after();
+    const uint32_t sQ = smem_u32(smem + L::kQD0 + st * L::kStage), sDO = sQ + L::kQTile;
+#pragma unroll
+    for (int kk = 0; kk < DK / 16; ++kk) {
+      uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
+      umma_bf16(tmem_base, desc_k(sK + oa), desc_k(sQ + ob), idesc_s, kk != 0);
+    }
+#pragma unroll
+    for (int kk = 0; kk < DK / 16; ++kk) {
+      uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
+      umma_bf16(tmem_base + 64, desc_k(sV + oa), desc_k(sDO + ob), idesc_s, kk != 0);
+    }
+    return true;
+  };
+  if (tid == 0 && t_begin < n_qt) {
+    ok = mbar_wait(bar_kv, 0, abort_flag, p.status, 31);
+    if (ok && issue_st(t_begin)) umma_commit(bar_m);
+  }
 
   for (int t = t_begin; t < n_qt && ok; ++t) {
     const int qb = t * 64;
     const uint32_t sQ = smem_u32(smem + L::kQD0 + (t & 1) * L::kStage), sDO = sQ + L::kQTile;
-    if (tid == 0) {
-      if (t + 1 < n_qt) load_qd(t + 1);
-      if (mbar_wait(&bar_qd[t & 1], ph_qd[t & 1], abort_flag, p.status, 32)) {
-        tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < DK / 16; ++kk) {
-          uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
-          umma_bf16(tmem_base, desc_k(sK + oa), desc_k(sQ + ob), idesc_s, kk != 0);
-        }
-#pragma unroll
-        for (int kk = 0; kk < DK / 16; ++kk) {
-          uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
-          umma_bf16(tmem_base + 64, desc_k(sV + oa), desc_k(sDO + ob), idesc_s, kk != 0);
-        }
-        umma_commit(bar_m);
-      }
-    }
-    ph_qd[t & 1] ^= 1;
     ok = mbar_wait(bar_m, ph_m, abort_flag, p.status, 33);
     ph_m ^= 1;
     if (!ok) break;
     tc_fence_after();
+    // the stage of tile t-1 is free (all MMAs that read it are done): fetch tile t+1 into it
+    if (tid == 0 && t > t_begin && t + 1 < n_qt) load_qd(t + 1);
     const int tcode = tile_code64(codes_s + qb, tid & 31);
     const bool fast = tcode > 0 && __all_sync(0xffffffffu, ck == tcode) &&
                       (!p.causal || k0 + (warp << 5) + 31 <= qb);           // warp-uniform: no mask needed
@@ -759,11 +771,12 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
       for (int ks = 0; ks < 4; ++ks)
         umma_bf16(tmem_base + 128 + DK, desc_k(sDSt + ks * 32), desc_mn(sQ + ks * 2048, 8192), idesc_acc,
                   first | ks);
-      umma_commit(bar_acc);
+      bool good = true;
+      if (t + 1 < n_qt) good = issue_st(t + 1);        // the scores of tile t are in registers by now
+      if (good) umma_commit(bar_m);
     }
-    ok = mbar_wait(bar_acc, ph_acc, abort_flag, p.status, 34);
-    ph_acc ^= 1;
   }
+  if (ok && t_begin < n_qt) ok = mbar_wait(bar_m, ph_m, abort_flag, p.status, 34);   // last accumulating MMAs done
 
   if (ok) {
     tc_fence_after();
@@ -926,6 +939,11 @@ bool attn_tc_supported(const AttnArgs& a) {
   if (a.ldq % 8 || a.ldk % 8 || a.ldv % 8 || a.ldo % 8) return false;
   if (a.O32 && (!al16(a.O32) || a.ldo32 % 4)) return false;
   if (a.causal && a.Tq != a.Tk) return false;
+  // every kernel's shared-memory footprint (tiles + distance-indexed windows) must fit one CTA
+  const int kSmemMax = 227 * 1024;
+  int need = a.dk == 64 ? max(FwdLayout<64>::bytes(a.Tk), max(DqLayout<64>::bytes(a.Tk), DkvLayout<64>::bytes(a.Tq)))
+                        : max(FwdLayout<128>::bytes(a.Tk), max(DqLayout<128>::bytes(a.Tk), DkvLayout<128>::bytes(a.Tq)));
+  if (need > kSmemMax) return false;
   return tc::get_encode() != nullptr;
 }
 

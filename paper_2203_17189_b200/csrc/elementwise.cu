@@ -195,14 +195,30 @@ __global__ void colsum_kernel(const float* __restrict__ partial, int n_part, int
 }
 
 // ------------------------------------------------------------------ gated GELU
+// FAST = true uses the hardware tanh approximation (relative error ~2^-11: below bfloat16 resolution);
+// the float32 validation mode keeps tanhf.
+template <bool FAST>
+__device__ __forceinline__ float tanh_sel(float x) {
+  if (FAST) {
+    float y;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+  }
+  return tanhf(x);
+}
+// gelu(u) and its derivative from one tanh
+template <bool FAST>
+__device__ __forceinline__ void gelu_both(float u, float& g, float& dg) {
+  const float c = 0.7978845608028654f, a = 0.044715f;
+  float u2 = u * u;
+  float t = tanh_sel<FAST>(c * (u + a * u * u2));
+  g = 0.5f * u * (1.f + t);
+  dg = 0.5f * (1.f + t) + 0.5f * u * (1.f - t * t) * c * (1.f + 3.f * a * u2);
+}
+template <bool FAST>
 __device__ __forceinline__ float gelu_tanh_f(float u) {
   const float c = 0.7978845608028654f, a = 0.044715f;
-  return 0.5f * u * (1.f + tanhf(c * (u + a * u * u * u)));
-}
-__device__ __forceinline__ float gelu_tanh_grad_f(float u) {
-  const float c = 0.7978845608028654f, a = 0.044715f;
-  float t = tanhf(c * (u + a * u * u * u));
-  return 0.5f * (1.f + t) + 0.5f * u * (1.f - t * t) * c * (1.f + 3.f * a * u * u);
+  return 0.5f * u * (1.f + tanh_sel<FAST>(c * (u + a * u * u * u)));
 }
 
 // h [rows, 2F] = [a | b]; hg = gelu(a) * b
@@ -213,8 +229,9 @@ __global__ void geglu_fwd_kernel(const T* __restrict__ h, T* __restrict__ hg, in
   if (idx >= (int64_t)rows * per_row) return;
   int r = (int)(idx / per_row), c = (int)(idx % per_row) << 2;
   float4 a = load4(h + (int64_t)r * 2 * F + c), b = load4(h + (int64_t)r * 2 * F + F + c);
-  store4(hg + (int64_t)r * F + c, make_float4(gelu_tanh_f(a.x) * b.x, gelu_tanh_f(a.y) * b.y,
-                                              gelu_tanh_f(a.z) * b.z, gelu_tanh_f(a.w) * b.w));
+  constexpr bool FAST = sizeof(T) == 2;
+  store4(hg + (int64_t)r * F + c, make_float4(gelu_tanh_f<FAST>(a.x) * b.x, gelu_tanh_f<FAST>(a.y) * b.y,
+                                              gelu_tanh_f<FAST>(a.z) * b.z, gelu_tanh_f<FAST>(a.w) * b.w));
 }
 // da = dhg * b * gelu'(a); db = dhg * gelu(a)
 template <typename T>
@@ -226,12 +243,12 @@ __global__ void geglu_bwd_kernel(const T* __restrict__ dhg, const T* __restrict_
   int r = (int)(idx / per_row), c = (int)(idx % per_row) << 2;
   float4 a = load4(h + (int64_t)r * 2 * F + c), b = load4(h + (int64_t)r * 2 * F + F + c);
   float4 g = load4(dhg + (int64_t)r * F + c);
-  store4(dh + (int64_t)r * 2 * F + c,
-         make_float4(g.x * b.x * gelu_tanh_grad_f(a.x), g.y * b.y * gelu_tanh_grad_f(a.y),
-                     g.z * b.z * gelu_tanh_grad_f(a.z), g.w * b.w * gelu_tanh_grad_f(a.w)));
-  store4(dh + (int64_t)r * 2 * F + F + c,
-         make_float4(g.x * gelu_tanh_f(a.x), g.y * gelu_tanh_f(a.y), g.z * gelu_tanh_f(a.z),
-                     g.w * gelu_tanh_f(a.w)));
+  constexpr bool FAST = sizeof(T) == 2;
+  float ge[4], dge[4];
+  gelu_both<FAST>(a.x, ge[0], dge[0]); gelu_both<FAST>(a.y, ge[1], dge[1]);
+  gelu_both<FAST>(a.z, ge[2], dge[2]); gelu_both<FAST>(a.w, ge[3], dge[3]);
+  store4(dh + (int64_t)r * 2 * F + c, make_float4(g.x * b.x * dge[0], g.y * b.y * dge[1], g.z * b.z * dge[2], g.w * b.w * dge[3]));
+  store4(dh + (int64_t)r * 2 * F + F + c, make_float4(g.x * ge[0], g.y * ge[1], g.z * ge[2], g.w * ge[3]));
 }
 
 // ------------------------------------------------------------------ cross-entropy + z-loss

@@ -168,6 +168,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int m0 = (tile % p.tiles_m) * BM, n0 = (tile / p.tiles_m) * BN;
       const int ab = it & 1;
       const uint32_t aph = (it >> 1) & 1;
+      if (p.out_f32 && (p.resid || p.accumulate)) {
+        // the float32 addend of this thread's row: pull its cache lines into L2 while the MMAs of the tile run
+        const int prow = m0 + quad * 32 + lane;
+        if (prow < p.M) {
+          const float* pr = p.resid ? p.resid + (int64_t)prow * p.ldr + n0 : (const float*)p.D + (int64_t)prow * p.ldd + n0;
+#pragma unroll
+          for (int c = 0; c < BN / 32; ++c)
+            if (n0 + c * 32 < p.N) asm volatile("prefetch.global.L2 [%0];" ::"l"(pr + c * 32));
+        }
+      }
       ok = mbar_wait(&tfull[ab], aph, abort_flag, p.status, 4);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -180,7 +190,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (col >= p.N) break;               // uniform across the warp
         uint32_t r[32];
         tmem_ld_32x32b_x32(tacc + c * 32, r);
-        tmem_wait_ld();
+        tmem_wait_ld_dep(r);
         if (row < p.M) {
           const bool full_chunk = col + 32 <= p.N;
           if (p.out_f32) {

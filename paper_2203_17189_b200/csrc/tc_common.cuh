@@ -26,10 +26,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n.reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n}"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"     // %3: suspend-time hint (ns): the
+      "selp.u32 %0, 1, 0, p;\n}"                                          // thread sleeps in hardware, not in a loop
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(20000u)
       : "memory");
   return ok != 0;
 }
