@@ -352,7 +352,7 @@ struct DqLayout {
 };
 
 template <int DK>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(256, DK == 64 ? 2 : 1)
 attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mdo,
                       const __grid_constant__ CUtensorMap mk, const __grid_constant__ CUtensorMap mv, TcParams p) {
   using L = DqLayout<DK>;
@@ -368,7 +368,8 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
   Bars* bars = (Bars*)(((uintptr_t)(codes_s + tkp) + 15) & ~(uintptr_t)15);
   volatile int* abort_flag = &bars->abort_flag;
 
-  const int tid = threadIdx.x, warp = tid >> 5;
+  // 256 threads: thread (row, half) owns tensor-memory lane `row` and one 32-column half of each score tile
+  const int tid = threadIdx.x, warp = tid >> 5, row = tid & 127, half = tid >> 7, quad = warp & 3;
   const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * 128;
   int n_kt = (p.Tk + 63) / 64;
   if (p.causal) n_kt = min(n_kt, (q0 + 127) / 64 + 1);
@@ -406,24 +407,24 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
   }
   if (warp == 0) tmem_alloc(&bars->tmem, kTmemCols);
   const int span = p.Tq + p.Tk - 1;
-  for (int w = tid; w < tkp + 128; w += 128) {
+  for (int w = tid; w < tkp + 128; w += 256) {
     int g = w - 127 - q0 + p.Tq - 1;
     bias_s[w] = (p.bias_delta && g >= 0 && g < span) ? p.bias_delta[(int64_t)h * span + g] * kLog2e : 0.f;
   }
-  for (int w = tid; w < 4 * wlen; w += 128) dbias_s[w] = 0.f;
-  for (int j = tid; j < tkp; j += 128) codes_s[j] = j < p.Tk ? p.code_k[b * p.Tk + j] : 0;
+  for (int w = tid; w < 4 * wlen; w += 256) dbias_s[w] = 0.f;
+  for (int j = tid; j < tkp; j += 256) codes_s[j] = j < p.Tk ? p.code_k[b * p.Tk + j] : 0;
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem;
   const uint32_t sQ = smem_u32(smem + L::kQ), sDO = smem_u32(smem + L::kDO), sDS = smem_u32(smem + L::kDS);
 
-  const int i = q0 + tid;
+  const int i = q0 + row;
   const bool row_in = i < p.Tq;
   const int cq = row_in ? p.code_q[b * p.Tq + i] : 0;
   const float lse2 = row_in ? p.lse[(int64_t)(b * p.H + h) * p.Tq + i] * kLog2e : -INFINITY;
   const float dl = row_in ? p.delta[(int64_t)(b * p.H + h) * p.Tq + i] : 0.f;
-  const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+  const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
   const float sc2 = p.scale * kLog2e;
   uint32_t ph_kv[3] = {0, 0, 0}, ph_m = 0;
   bool ok = true;
@@ -463,25 +464,22 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
     if (tid == 0 && t + 2 < n_kt) load_kv(t + 2);      // its stage held tile t-1, whose MMAs are all done
     const int tcode = tile_code64(codes_s + k0, tid & 31);
     const bool fast = tcode > 0 && __all_sync(0xffffffffu, cq == tcode) &&
-                      (!p.causal || k0 + 63 <= q0 + (warp << 5));           // warp-uniform: no mask needed
-    const float* brow = bias_s + (k0 - tid + 127);
+                      (!p.causal || k0 + 63 <= q0 + (quad << 5));           // warp-uniform: no mask needed
+    const float* brow = bias_s + (k0 - row + 127);
     const int lane = tid & 31;
-    float* dbwin = dbias_s + warp * wlen + k0;        // this warp's window; entry = key - (row in warp) + 31
+    float* dbwin = dbias_s + quad * wlen + k0;        // window of this row quarter; entry = key - (row in quarter) + 31
     const bool has_bias = p.bias_delta != nullptr;
-    uint32_t rs[2][32], rp[2][32];
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, rs[c]);
-      tmem_ld_32x32b_x32(tmem_base + lane_off + 64 + c * 32, rp[c]);
-    }
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      tmem_wait_ld_dep(rs[c]);
-      tmem_wait_ld_dep(rp[c]);
+    uint32_t rs[32], rp[32];
+    const int c = half;                                // this thread's 32 keys of the tile
+    tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, rs);
+    tmem_ld_32x32b_x32(tmem_base + lane_off + 64 + c * 32, rp);
+    tmem_wait_ld_dep(rs);
+    tmem_wait_ld_dep(rp);
+    {
       float ds[32];
 #pragma unroll
       for (int jj = 0; jj < 32; ++jj) {
-        float sv = has_bias ? fmaf(__uint_as_float(rs[c][jj]), sc2, brow[c * 32 + jj]) : __uint_as_float(rs[c][jj]) * sc2;
+        float sv = has_bias ? fmaf(__uint_as_float(rs[jj]), sc2, brow[c * 32 + jj]) : __uint_as_float(rs[jj]) * sc2;
         float pr = ex2_approx(sv - lse2);
         if (!fast) {
           int j = k0 + c * 32 + jj;
@@ -489,22 +487,20 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
           bool valid = ck != 0 && ck == cq && (!p.causal || j <= i) && lse2 != -INFINITY;
           pr = valid ? pr : 0.f;
         }
-        ds[jj] = pr * (__uint_as_float(rp[c][jj]) - dl);
+        ds[jj] = pr * (__uint_as_float(rp[jj]) - dl);
       }
       if (want_db) {
-        // Diagonal sums of this warp's 32 x 32 block without atomics: at step t lane l takes column t of
-        // row (l + t) mod 32, which lies on diagonal (col - row) = -l when l + t < 32 and 32 - l otherwise.
+        // Diagonal sums of this warp's 32 x 32 block: at step t lane l takes column t of row (l + t) mod 32,
+        // which lies on diagonal (col - row) = -l when l + t < 32 and 32 - l otherwise.
         float a0 = 0.f, a1 = 0.f;
 #pragma unroll
-        for (int t = 0; t < 32; ++t) {
-          float v = __shfl_sync(0xffffffffu, ds[t], (lane + t) & 31);
-          if (lane + t < 32) a0 += v; else a1 += v;
+        for (int t2 = 0; t2 < 32; ++t2) {
+          float v = __shfl_sync(0xffffffffu, ds[t2], (lane + t2) & 31);
+          if (lane + t2 < 32) a0 += v; else a1 += v;
         }
-        // window entry (col - row + 31): diagonal -l -> 31 - l, diagonal 32 - l -> 63 - l; distinct per lane
-        dbwin[c * 32 + 31 - lane] += a0;
-        __syncwarp();
-        dbwin[c * 32 + 63 - lane] += a1;
-        __syncwarp();
+        // window entry (col - row + 31); the two column halves of a row quarter overlap there: atomics
+        atomicAdd(&dbwin[c * 32 + 31 - lane], a0);
+        atomicAdd(&dbwin[c * 32 + 63 - lane], a1);
       }
 #pragma unroll
       for (int q8 = 0; q8 < 4; ++q8) {
@@ -513,7 +509,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
         v.y = pack_bf16(ds[q8 * 8 + 2], ds[q8 * 8 + 3]);
         v.z = pack_bf16(ds[q8 * 8 + 4], ds[q8 * 8 + 5]);
         v.w = pack_bf16(ds[q8 * 8 + 6], ds[q8 * 8 + 7]);
-        store_swizzled_16B(smem + L::kDS, tid, c * 4 + q8, v);
+        store_swizzled_16B(smem + L::kDS, row, c * 4 + q8, v);
       }
     }
     fence_proxy_async();
@@ -534,12 +530,12 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
 
   if (ok) {
     tc_fence_after();
-    bf16* drow = (bf16*)p.out0 + (int64_t)(b * p.Tq + i) * p.ld0 + h * DK;
+    bf16* drow = (bf16*)p.out0 + (int64_t)(b * p.Tq + i) * p.ld0 + h * DK + half * (DK / 2);
 #pragma unroll
-    for (int c = 0; c < DK / 32; ++c) {
+    for (int c = 0; c < DK / 64; ++c) {
       uint32_t r[32];
-      tmem_ld_32x32b_x32(tmem_base + lane_off + 128 + c * 32, r);
-      tmem_wait_ld();
+      tmem_ld_32x32b_x32(tmem_base + lane_off + 128 + half * (DK / 2) + c * 32, r);
+      tmem_wait_ld_dep(r);
       if (row_in) {
 #pragma unroll
         for (int d = 0; d < 32; d += 8) {
@@ -561,7 +557,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
   __syncthreads();
   if (ok && want_db) {
     // CTA-level index (key - row + 127) = warp-level index + 96 - 32 * warp
-    for (int w = tid; w < tkp + 128; w += 128) {
+    for (int w = tid; w < tkp + 128; w += 256) {
       float v = 0.f;
 #pragma unroll
       for (int wp = 0; wp < 4; ++wp) {
@@ -594,21 +590,22 @@ struct DkvLayout {
 };
 
 template <int DK>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(256, DK == 64 ? 2 : 1)
 attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mdo,
                        const __grid_constant__ CUtensorMap mk, const __grid_constant__ CUtensorMap mv, TcParams p) {
   using L = DkvLayout<DK>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int tqp = (p.Tq + 63) / 64 * 64;
-  float* bias_s = (float*)(smem + L::kMisc);          // [tqp + 128], indexed by (tid - i_local + tqp... see below)
+  float* bias_s = (float*)(smem + L::kMisc);          // [tqp + 128], entry (key row - query + tqp), log2 units
   float* lse_s = bias_s + tqp + 128;                  // [tqp]  (log2 units)
   float* dl_s = lse_s + tqp;                          // [tqp]
   int* codes_s = (int*)(dl_s + tqp);                  // [tqp] query codes
   Bars* bars = (Bars*)(((uintptr_t)(codes_s + tqp) + 15) & ~(uintptr_t)15);
   volatile int* abort_flag = &bars->abort_flag;
 
-  const int tid = threadIdx.x, warp = tid >> 5;
+  // 256 threads: thread (row, half) owns tensor-memory lane `row` (a key) and 32 of the 64 queries of each tile
+  const int tid = threadIdx.x, warp = tid >> 5, row = tid & 127, half = tid >> 7, quad = warp & 3;
   const int b = blockIdx.z, h = blockIdx.y, k0 = blockIdx.x * 128;
   const int n_qt = (p.Tq + 63) / 64;
   const int t_begin = p.causal ? k0 / 64 : 0;          // queries before k0 see none of these keys
@@ -645,12 +642,12 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
   }
   if (warp == 0) tmem_alloc(&bars->tmem, kTmemCols);
   const int span = p.Tq + p.Tk - 1;
-  // distance of (key j = k0 + tid, query i): j - i ; window index w = tid - i + tqp  in [1, tqp + 127]
-  for (int w = tid; w < tqp + 128; w += 128) {
+  // distance of (key j = k0 + row, query i): j - i ; window index w = row - i + tqp  in [1, tqp + 127]
+  for (int w = tid; w < tqp + 128; w += 256) {
     int g = (w - tqp) + k0 + p.Tq - 1;
     bias_s[w] = (p.bias_delta && g >= 0 && g < span) ? p.bias_delta[(int64_t)h * span + g] * kLog2e : 0.f;
   }
-  for (int q = tid; q < tqp; q += 128) {
+  for (int q = tid; q < tqp; q += 256) {
     bool in = q < p.Tq;
     lse_s[q] = in ? p.lse[(int64_t)(b * p.H + h) * p.Tq + q] * kLog2e : -INFINITY;
     dl_s[q] = in ? p.delta[(int64_t)(b * p.H + h) * p.Tq + q] : 0.f;
@@ -662,10 +659,10 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
   const uint32_t tmem_base = bars->tmem;
   const uint32_t sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV), sPt = smem_u32(smem + L::kPt),
                  sDSt = smem_u32(smem + L::kDSt);
-  const int j = k0 + tid;
+  const int j = k0 + row;
   const bool row_in = j < p.Tk;
   const int ck = row_in ? p.code_k[b * p.Tk + j] : 0;
-  const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+  const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
   const float sc2 = p.scale * kLog2e;
   uint32_t ph_qd[2] = {0, 0}, ph_m = 0;
   bool ok = true;
@@ -706,21 +703,16 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
     if (tid == 0 && t > t_begin && t + 1 < n_qt) load_qd(t + 1);
     const int tcode = tile_code64(codes_s + qb, tid & 31);
     const bool fast = tcode > 0 && __all_sync(0xffffffffu, ck == tcode) &&
-                      (!p.causal || k0 + (warp << 5) + 31 <= qb);           // warp-uniform: no mask needed
-    const float* brow = bias_s + (tid - qb + tqp);       // element q of the tile: brow[-(q - qb)]
+                      (!p.causal || k0 + (quad << 5) + 31 <= qb);           // warp-uniform: no mask needed
+    const float* brow = bias_s + (row - qb + tqp);       // element q of the tile: brow[-(q - qb)]
     const bool has_bias = p.bias_delta != nullptr;
-    uint32_t rsa[2][32], rpa[2][32];
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, rsa[c]);
-      tmem_ld_32x32b_x32(tmem_base + lane_off + 64 + c * 32, rpa[c]);
-    }
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      uint32_t (&rs)[32] = rsa[c];
-      uint32_t (&rp)[32] = rpa[c];
-      tmem_wait_ld_dep(rs);
-      tmem_wait_ld_dep(rp);
+    uint32_t rs[32], rp[32];
+    const int c = half;                                // this thread's 32 queries of the tile
+    tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, rs);
+    tmem_ld_32x32b_x32(tmem_base + lane_off + 64 + c * 32, rp);
+    tmem_wait_ld_dep(rs);
+    tmem_wait_ld_dep(rp);
+    {
       float pt[32], ds[32];
 #pragma unroll
       for (int i4 = 0; i4 < 8; ++i4) {
@@ -750,12 +742,12 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
         v.y = pack_bf16(pt[q8 * 8 + 2], pt[q8 * 8 + 3]);
         v.z = pack_bf16(pt[q8 * 8 + 4], pt[q8 * 8 + 5]);
         v.w = pack_bf16(pt[q8 * 8 + 6], pt[q8 * 8 + 7]);
-        store_swizzled_16B(smem + L::kPt, tid, c * 4 + q8, v);
+        store_swizzled_16B(smem + L::kPt, row, c * 4 + q8, v);
         v.x = pack_bf16(ds[q8 * 8 + 0], ds[q8 * 8 + 1]);
         v.y = pack_bf16(ds[q8 * 8 + 2], ds[q8 * 8 + 3]);
         v.z = pack_bf16(ds[q8 * 8 + 4], ds[q8 * 8 + 5]);
         v.w = pack_bf16(ds[q8 * 8 + 6], ds[q8 * 8 + 7]);
-        store_swizzled_16B(smem + L::kDSt, tid, c * 4 + q8, v);
+        store_swizzled_16B(smem + L::kDSt, row, c * 4 + q8, v);
       }
     }
     fence_proxy_async();
@@ -780,16 +772,17 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
 
   if (ok) {
     tc_fence_after();
-    bf16* krow = (bf16*)p.out0 + (int64_t)(b * p.Tk + j) * p.ld0 + h * DK;
-    bf16* vrow = (bf16*)p.out1 + (int64_t)(b * p.Tk + j) * p.ld1 + h * DK;
+    bf16* krow = (bf16*)p.out0 + (int64_t)(b * p.Tk + j) * p.ld0 + h * DK + half * (DK / 2);
+    bf16* vrow = (bf16*)p.out1 + (int64_t)(b * p.Tk + j) * p.ld1 + h * DK + half * (DK / 2);
     const bool any = t_begin < n_qt;
 #pragma unroll
-    for (int c = 0; c < DK / 32; ++c) {
+    for (int c = 0; c < DK / 64; ++c) {
       uint32_t rv[32], rk[32];
       if (any) {
-        tmem_ld_32x32b_x32(tmem_base + lane_off + 128 + c * 32, rv);
-        tmem_ld_32x32b_x32(tmem_base + lane_off + 128 + DK + c * 32, rk);
-        tmem_wait_ld();
+        tmem_ld_32x32b_x32(tmem_base + lane_off + 128 + half * (DK / 2) + c * 32, rv);
+        tmem_ld_32x32b_x32(tmem_base + lane_off + 128 + DK + half * (DK / 2) + c * 32, rk);
+        tmem_wait_ld_dep(rv);
+        tmem_wait_ld_dep(rk);
       } else {
 #pragma unroll
         for (int d = 0; d < 32; ++d) rv[d] = rk[d] = 0u;
@@ -909,7 +902,7 @@ cudaError_t bwd_launch(const AttnArgs& a, int* status, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     p.out0 = a.dQ; p.ld0 = a.lddq;
     dim3 grid((a.Tq + 127) / 128, a.H, a.B);
-    attn_bwd_dq_tc_kernel<DK><<<grid, 128, smem, st>>>(mq, mdo, mk, mv, p);
+    attn_bwd_dq_tc_kernel<DK><<<grid, 256, smem, st>>>(mq, mdo, mk, mv, p);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
@@ -923,7 +916,7 @@ cudaError_t bwd_launch(const AttnArgs& a, int* status, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     p.out0 = a.dK; p.ld0 = a.lddk; p.out1 = a.dV; p.ld1 = a.lddv;
     dim3 grid((a.Tk + 127) / 128, a.H, a.B);
-    attn_bwd_dkv_tc_kernel<DK><<<grid, 128, smem, st>>>(mq, mdo, mk, mv, p);
+    attn_bwd_dkv_tc_kernel<DK><<<grid, 256, smem, st>>>(mq, mdo, mk, mv, p);
     e = cudaGetLastError();
   }
   return e;
