@@ -46,7 +46,9 @@ struct Smem {
   static constexpr int kBBytes = BN * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kBarOffset = STAGES * kStageBytes;
-  static constexpr int kTotal = kBarOffset + 256 + 1024;   // barriers + slack for 1024-byte alignment
+  static constexpr int kEpiOffset = kBarOffset + 256;       // 4 epilogue warps x [32][36] floats (transpose buffers)
+  static constexpr int kEpiBytes = 4 * 32 * 36 * 4;
+  static constexpr int kTotal = kEpiOffset + kEpiBytes + 1024;   // + slack for 1024-byte alignment
 };
 
 template <int BN, int STAGES, bool A_MN, bool B_MN>
@@ -168,76 +170,67 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int m0 = (tile % p.tiles_m) * BM, n0 = (tile / p.tiles_m) * BN;
       const int ab = it & 1;
       const uint32_t aph = (it >> 1) & 1;
-      if (p.out_f32 && (p.resid || p.accumulate)) {
-        // the float32 addend of this thread's row: pull its cache lines into L2 while the MMAs of the tile run
-        const int prow = m0 + quad * 32 + lane;
-        if (prow < p.M) {
-          const float* pr = p.resid ? p.resid + (int64_t)prow * p.ldr + n0 : (const float*)p.D + (int64_t)prow * p.ldd + n0;
-#pragma unroll
-          for (int c = 0; c < BN / 32; ++c)
-            if (n0 + c * 32 < p.N) asm volatile("prefetch.global.L2 [%0];" ::"l"(pr + c * 32));
-        }
-      }
       ok = mbar_wait(&tfull[ab], aph, abort_flag, p.status, 4);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const int row = m0 + quad * 32 + lane;
       const uint32_t tacc = tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16);
+      // Each thread holds one accumulator row; going through a per-warp shared-memory tile turns the stores
+      // (and the loads of the float32 addend) into 128-byte row segments instead of 32 scattered pieces.
+      float* tbuf = reinterpret_cast<float*>(smem + S::kEpiOffset) + quad * (32 * 36);
+      const int rr0 = lane >> 3, cc = (lane & 7) * 4;
+      // float32 addend (residual input, or D itself when accumulating), fetched one chunk ahead of its use
+      const float* addend = !p.out_f32 ? nullptr : (p.resid ? p.resid : (p.accumulate ? (const float*)p.D : nullptr));
+      const int ld_add = p.resid ? p.ldr : p.ldd;
+      float4 add_next[8];
+      auto fetch_addend = [&](int c, float4 (&dst)[8]) {
+        const int col = n0 + c * 32 + cc;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int row = m0 + quad * 32 + i * 4 + rr0;
+          dst[i] = (addend && row < p.M && col < p.N) ? *reinterpret_cast<const float4*>(addend + (int64_t)row * ld_add + col)
+                                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      };
+      fetch_addend(0, add_next);
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
-        const int col = n0 + c * 32;
-        if (col >= p.N) break;               // uniform across the warp
+        const int col0 = n0 + c * 32;
+        if (col0 >= p.N) break;               // uniform across the warp
+        float4 add_cur[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) add_cur[i] = add_next[i];
         uint32_t r[32];
         tmem_ld_32x32b_x32(tacc + c * 32, r);
         tmem_wait_ld_dep(r);
-        if (row < p.M) {
-          const bool full_chunk = col + 32 <= p.N;
-          if (p.out_f32) {
-            float* d = (float*)p.D + (int64_t)row * p.ldd + col;
-            const float* rs = p.resid ? p.resid + (int64_t)row * p.ldr + col : (p.accumulate ? d : nullptr);
-            if (full_chunk) {
 #pragma unroll
-              for (int j = 0; j < 32; j += 4) {
-                float4 v = make_float4(p.alpha * __uint_as_float(r[j]), p.alpha * __uint_as_float(r[j + 1]),
-                                       p.alpha * __uint_as_float(r[j + 2]), p.alpha * __uint_as_float(r[j + 3]));
-                if (rs) {
-                  float4 a = *reinterpret_cast<const float4*>(rs + j);
-                  v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
-                }
-                *reinterpret_cast<float4*>(d + j) = v;
-              }
+        for (int j = 0; j < 8; ++j)
+          *reinterpret_cast<float4*>(tbuf + lane * 36 + j * 4) =
+              make_float4(p.alpha * __uint_as_float(r[4 * j]), p.alpha * __uint_as_float(r[4 * j + 1]),
+                          p.alpha * __uint_as_float(r[4 * j + 2]), p.alpha * __uint_as_float(r[4 * j + 3]));
+        __syncwarp();
+        if (addend && c + 1 < BN / 32) fetch_addend(c + 1, add_next);     // in flight while this chunk is stored
+        const int col = col0 + cc;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int rr = i * 4 + rr0;
+          const int row = m0 + quad * 32 + rr;
+          float4 v = *reinterpret_cast<const float4*>(tbuf + rr * 36 + cc);
+          if (row < p.M && col < p.N) {        // N is a multiple of 4: a float4 never straddles the edge
+            if (p.out_f32) {
+              v.x += add_cur[i].x; v.y += add_cur[i].y; v.z += add_cur[i].z; v.w += add_cur[i].w;
+              *reinterpret_cast<float4*>((float*)p.D + (int64_t)row * p.ldd + col) = v;
             } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                if (col + j < p.N) {
-                  float v = p.alpha * __uint_as_float(r[j]);
-                  if (rs) v += rs[j];
-                  d[j] = v;
-                }
-              }
-            }
-          } else {
-            bf16* d = (bf16*)p.D + (int64_t)row * p.ldd + col;
-            if (full_chunk) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                uint4 o;
-                __nv_bfloat162 b0 = __floats2bfloat162_rn(p.alpha * __uint_as_float(r[j]), p.alpha * __uint_as_float(r[j + 1]));
-                __nv_bfloat162 b1 = __floats2bfloat162_rn(p.alpha * __uint_as_float(r[j + 2]), p.alpha * __uint_as_float(r[j + 3]));
-                __nv_bfloat162 b2 = __floats2bfloat162_rn(p.alpha * __uint_as_float(r[j + 4]), p.alpha * __uint_as_float(r[j + 5]));
-                __nv_bfloat162 b3 = __floats2bfloat162_rn(p.alpha * __uint_as_float(r[j + 6]), p.alpha * __uint_as_float(r[j + 7]));
-                o.x = *reinterpret_cast<uint32_t*>(&b0); o.y = *reinterpret_cast<uint32_t*>(&b1);
-                o.z = *reinterpret_cast<uint32_t*>(&b2); o.w = *reinterpret_cast<uint32_t*>(&b3);
-                *reinterpret_cast<uint4*>(d + j) = o;
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (col + j < p.N) d[j] = __float2bfloat16_rn(p.alpha * __uint_as_float(r[j]));
+              bf16* d = (bf16*)p.D + (int64_t)row * p.ldd + col;
+              __nv_bfloat162 b0 = __floats2bfloat162_rn(v.x, v.y), b1 = __floats2bfloat162_rn(v.z, v.w);
+              uint2 o;
+              o.x = *reinterpret_cast<uint32_t*>(&b0);
+              o.y = *reinterpret_cast<uint32_t*>(&b1);
+              *reinterpret_cast<uint2*>(d) = o;
             }
           }
         }
+        __syncwarp();                          // the tile is rewritten by the next chunk
       }
       tc_fence_before();
       __syncwarp();
@@ -312,6 +305,7 @@ bool gemm_tc_supported(const GemmArgs& g) {
   if (!al16(g.A) || !al16(g.B) || !al16(g.D)) return false;
   if (g.lda % 8 || g.ldb % 8) return false;
   if (g.out_f32 ? (g.ldd % 4) : (g.ldd % 8)) return false;
+  if (g.N % 4) return false;
   if (g.resid && (!al16(g.resid) || g.ldr % 4)) return false;
   if (g.accumulate && !g.out_f32) return false;
   return tc::get_encode() != nullptr;
