@@ -186,11 +186,13 @@ T5_API int t5_xent_zloss(int32_t dtype, void* d_logits, const int32_t* d_targets
 /* D[M,N] = alpha * A * B (+ D when accumulate), bf16/f32 operands, f32 accumulation.
  * a_kmajor: A is stored [M,K] (else [K,M]); b_kmajor: B is stored [N,K] (else [K,N]);
  * lda/ldb/ldd are row strides in elements.  out_f32: D is float32, else the operand
- * dtype.  impl 0 = SIMT kernel, 1 = tcgen05/TMEM/TMA kernel (bfloat16 only). */
+ * dtype.  impl 0 = SIMT kernel, 1 = tcgen05/TMEM/TMA kernel (bfloat16 only).
+ * d_sk_flags: NULL, or 160 zeroed int32 that allow the tcgen05 kernel to cut the
+ * tiles of a partial last wave along K over all SMs (float32 output only). */
 T5_API int t5_gemm(int32_t dtype, int32_t impl, int32_t M, int32_t N, int32_t K, float alpha,
             const void* d_A, int32_t lda, int32_t a_kmajor, const void* d_B, int32_t ldb,
             int32_t b_kmajor, void* d_D, int32_t ldd, int32_t out_f32, int32_t accumulate,
-            void* stream);
+            int32_t* d_sk_flags, void* stream);
 
 /* One attention call on raw buffers (forward, or backward given the forward's
  * outputs):  S_ij = scale q_i.k_j + bias_delta[h, j - i + Tq - 1], masked by

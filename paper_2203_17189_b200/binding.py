@@ -81,7 +81,7 @@ def lib():
         L.t5_launch_count.argtypes = [vp, C.POINTER(i64)]
         L.t5_relpos_buckets.argtypes = [i32, i32, i32, i32, i32, vp, vp]
         L.t5_xent_zloss.argtypes = [i32, vp, vp, i32, i32, f32, vp, vp, vp, vp]
-        L.t5_gemm.argtypes = [i32, i32, i32, i32, i32, f32, vp, i32, i32, vp, i32, i32, vp, i32, i32, i32, vp]
+        L.t5_gemm.argtypes = [i32, i32, i32, i32, i32, f32, vp, i32, i32, vp, i32, i32, vp, i32, i32, i32, vp, vp]
         L.t5_attention.argtypes = ([i32] * 9 + [f32] + [vp, i32] * 3 + [vp, i32, vp, vp, vp, vp, vp]
                                    + [vp, i32] * 4 + [vp, vp, vp])
         L.t5_attention_backward_noalloc.argtypes = ([i32] * 8 + [f32] + [vp, i32] * 4 + [vp] * 5
@@ -237,11 +237,11 @@ def t5_xent_zloss(logits, targets, z_loss, W, sums, lse):
                                _ptr(lse), _stream()))
 
 
-def t5_gemm(impl, M, N, K, alpha, A, lda, a_kmajor, B, ldb, b_kmajor, D, ldd, accumulate=False):
+def t5_gemm(impl, M, N, K, alpha, A, lda, a_kmajor, B, ldb, b_kmajor, D, ldd, accumulate=False, sk_flags=None):
     dtype = 0 if A.dtype == torch.float32 else 1
     out_f32 = int(D.dtype == torch.float32)
     _check(lib().t5_gemm(dtype, impl, M, N, K, alpha, _ptr(A), lda, int(a_kmajor), _ptr(B), ldb,
-                         int(b_kmajor), _ptr(D), ldd, out_f32, int(accumulate), _stream()))
+                         int(b_kmajor), _ptr(D), ldd, out_f32, int(accumulate), _ptr(sk_flags), _stream()))
 
 
 def t5_attention(impl, backward, B, H, Tq, Tk, d_kv, causal, scale, q, k, v, o, lse, code_q, code_k, bias_delta,

@@ -62,6 +62,8 @@ struct GemmArgs {
   void* D; int ldd; int out_f32;          // D[M,N]; float32 or operand dtype
   const float* resid; int ldr;            // optional float32 addend (D may alias it)
   int accumulate;                         // D += (float32 output only)
+  int* sk_flags;                          // optional: >= 160 zeroed ints; lets the tcgen05 kernel split the
+                                          // tiles of a partial last wave along K over all SMs (float32 output)
 };
 cudaError_t gemm_simt(int dtype, const GemmArgs& g, cudaStream_t st);
 // tcgen05 path: bf16 operands only.  `status` is a device int set non-zero if a

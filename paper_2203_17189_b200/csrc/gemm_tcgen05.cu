@@ -38,6 +38,48 @@ struct Params {
   int accumulate;
   int tiles_m, tiles_n;
   int* status;
+  // stream-K tail: the first sk_full * gridDim.x tiles are walked tile by tile; the remaining sk_rem tiles
+  // (a partial wave) are cut along K into gridDim.x equal ranges of k-blocks.  sk_rem = 0 turns it off.
+  int sk_full, sk_rem;
+  int* sk_flags;      // [sk_rem], zeroed: counts the epilogue warps of the storing segment that are done
+};
+
+// One unit of work of a CTA: k-blocks [kb0, kb1) of a tile.
+//   kind 0: the whole tile;  1: the segment that reaches the tile's last k-block (it stores, then raises
+//   the tile's flag);  2: an earlier segment (waits for the flag, then adds atomically).
+struct Work { int tile, kb0, kb1, kind, flag; };
+
+struct WorkIter {
+  int it = 0;
+  int n_tiles, k_blocks, sk_full, sk_rem;
+  long long cur, u1;
+  __device__ WorkIter(const Params& p, int kb) : n_tiles(p.tiles_m * p.tiles_n), k_blocks(kb), sk_full(p.sk_full), sk_rem(p.sk_rem) {
+    long long U = (long long)sk_rem * kb;
+    cur = U * blockIdx.x / gridDim.x;
+    u1 = U * (blockIdx.x + 1) / gridDim.x;
+  }
+  __device__ bool next(Work& w) {
+    if (sk_rem == 0) {
+      int tile = blockIdx.x + it * gridDim.x;
+      if (tile >= n_tiles) return false;
+      w = {tile, 0, k_blocks, 0, 0};
+      ++it;
+      return true;
+    }
+    if (it < sk_full) {
+      w = {(int)(blockIdx.x + it * gridDim.x), 0, k_blocks, 0, 0};
+      ++it;
+      return true;
+    }
+    if (cur >= u1) return false;
+    int t = (int)(cur / k_blocks), kb0 = (int)(cur % k_blocks);
+    long long left = u1 - cur;
+    int kb1 = left < k_blocks - kb0 ? kb0 + (int)left : k_blocks;
+    cur += kb1 - kb0;
+    w = {sk_full * (int)gridDim.x + t, kb0, kb1, (kb0 == 0 && kb1 == k_blocks) ? 0 : (kb1 == k_blocks ? 1 : 2), t};
+    ++it;
+    return true;
+  }
 };
 
 template <int BN, int STAGES>
@@ -91,9 +133,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
       for (int i = 0; i < STAGES; ++i) issued[i] = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile % p.tiles_m) * BM, n0 = (tile / p.tiles_m) * BN;
-        for (int kb = 0; kb < k_blocks; ++kb) {
+      WorkIter wi(p, k_blocks);
+      Work w;
+      while (ok && wi.next(w)) {
+        const int m0 = (w.tile % p.tiles_m) * BM, n0 = (w.tile / p.tiles_m) * BN;
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status, 1)) { ok = false; break; }
           unsigned char* sa = smem + s * S::kStageBytes;
           unsigned char* sb = sa + S::kABytes;
@@ -136,13 +180,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       uint32_t ph = 0;
       int it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
+      WorkIter wi(p, k_blocks);
+      Work w;
+      for (; ok && wi.next(w); ++it) {
         const int ab = it & 1;
         const uint32_t aph = (it >> 1) & 1;
         if (!mbar_wait(&tempty[ab], aph ^ 1, abort_flag, p.status, 2)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tacc = tmem_base + ab * BN;
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait(&full[s], ph, abort_flag, p.status, 3)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + s * S::kStageBytes);
@@ -153,7 +199,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // MN-major: 16 K-rows = two 8-row groups of 1024 bytes further.
             uint64_t da = A_MN ? make_desc(sa + k * 2048, 8192, 1024) : make_desc(sa + k * 32, 16, 1024);
             uint64_t db = B_MN ? make_desc(sb + k * 2048, 8192, 1024) : make_desc(sb + k * 32, 16, 1024);
-            umma_bf16(tacc, da, db, idesc, (kb | k) != 0);
+            umma_bf16(tacc, da, db, idesc, ((kb - w.kb0) | k) != 0);
           }
           umma_commit(&empty[s]);
           if (++s == STAGES) { s = 0; ph ^= 1; }
@@ -166,21 +212,39 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int quad = warp & 3;
     int it = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
-      const int m0 = (tile % p.tiles_m) * BM, n0 = (tile / p.tiles_m) * BN;
+    WorkIter wi(p, k_blocks);
+    Work w;
+    for (; ok && wi.next(w); ++it) {
+      const int m0 = (w.tile % p.tiles_m) * BM, n0 = (w.tile / p.tiles_m) * BN;
       const int ab = it & 1;
       const uint32_t aph = (it >> 1) & 1;
       ok = mbar_wait(&tfull[ab], aph, abort_flag, p.status, 4);
+      if (ok && w.kind == 2) {
+        // an earlier K-segment of a split tile: the segment that stores must be done first
+        volatile int* flag = p.sk_flags + w.flag;
+        long long t0 = clock64();
+        while (*flag < 4) {
+          if (clock64() - t0 > kWaitCycles) {
+            if (p.status) atomicCAS(p.status, 0, 5);
+            ok = false;
+            break;
+          }
+          __nanosleep(200);
+        }
+        __threadfence();
+      }
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
+      const bool add_atomic = w.kind == 2;
       const uint32_t tacc = tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16);
       // Each thread holds one accumulator row; going through a per-warp shared-memory tile turns the stores
       // (and the loads of the float32 addend) into 128-byte row segments instead of 32 scattered pieces.
       float* tbuf = reinterpret_cast<float*>(smem + S::kEpiOffset) + quad * (32 * 36);
       const int rr0 = lane >> 3, cc = (lane & 7) * 4;
       // float32 addend (residual input, or D itself when accumulating), fetched one chunk ahead of its use
-      const float* addend = !p.out_f32 ? nullptr : (p.resid ? p.resid : (p.accumulate ? (const float*)p.D : nullptr));
+      const float* addend = (!p.out_f32 || add_atomic) ? nullptr
+                                                        : (p.resid ? p.resid : (p.accumulate ? (const float*)p.D : nullptr));
       const int ld_add = p.resid ? p.ldr : p.ldd;
       float4 add_next[8];
       auto fetch_addend = [&](int c, float4 (&dst)[8]) {
@@ -217,7 +281,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int row = m0 + quad * 32 + rr;
           float4 v = *reinterpret_cast<const float4*>(tbuf + rr * 36 + cc);
           if (row < p.M && col < p.N) {        // N is a multiple of 4: a float4 never straddles the edge
-            if (p.out_f32) {
+            if (add_atomic) {
+              float* d = (float*)p.D + (int64_t)row * p.ldd + col;
+              asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(d), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+                           : "memory");
+            } else if (p.out_f32) {
               v.x += add_cur[i].x; v.y += add_cur[i].y; v.z += add_cur[i].z; v.w += add_cur[i].w;
               *reinterpret_cast<float4*>((float*)p.D + (int64_t)row * p.ldd + col) = v;
             } else {
@@ -231,6 +299,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
         }
         __syncwarp();                          // the tile is rewritten by the next chunk
+      }
+      if (w.kind == 1) {          // publish this warp's part of the stored tile to the adding segments
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) atomicAdd(p.sk_flags + w.flag, 1);
       }
       tc_fence_before();
       __syncwarp();
@@ -279,6 +352,17 @@ cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& 
   p.tiles_m = (g.M + BM - 1) / BM; p.tiles_n = (g.N + BN - 1) / BN; p.status = status;
   int tiles = p.tiles_m * p.tiles_n;
   int grid = tiles < g_num_sms ? tiles : g_num_sms;
+  p.sk_full = 0; p.sk_rem = 0; p.sk_flags = nullptr;
+  const int k_blocks = (g.K + BK - 1) / BK;
+  const int rem = tiles % g_num_sms;
+  // split the tiles of a partial last wave along K when that wave would leave a good part of the GPU idle
+  // (measured: pays only for long K and after at least one full wave; short-K tiles lose more in the extra
+  // atomic epilogues than the idle SMs cost)
+  if (g.sk_flags && g.out_f32 && rem > 0 && k_blocks >= 128 && tiles >= g_num_sms && g_num_sms <= 160 &&
+      (g_num_sms - rem) * 8 > g_num_sms * (tiles / g_num_sms + 1)) {
+    grid = g_num_sms;
+    p.sk_full = tiles / g_num_sms; p.sk_rem = rem; p.sk_flags = g.sk_flags;
+  }
   kern<<<grid, kThreads, S::kTotal, st>>>(ma, mb, p);
   return cudaGetLastError();
 }

@@ -36,7 +36,7 @@ struct Workspace {
   float *enc_x_final, *enc_rstd_f, *dec_x_final, *dec_rstd_f;
   void *enc_out, *dec_z, *logits;
   float* lse_tok;
-  int *enc_code, *dec_code, *dec_in, *W_int, *status;
+  int *enc_code, *dec_code, *dec_in, *W_int, *status, *sk_flags;
   float* W_f;
   double* sums;
   float *bias_enc, *bias_dec, *dbias_enc, *dbias_dec, *norm_partial, *delta;
@@ -46,6 +46,7 @@ struct Workspace {
 };
 
 char g_create_error[256] = "";
+constexpr int kSkSlices = 2048, kSkSliceInts = 160;
 
 }  // namespace
 
@@ -190,6 +191,7 @@ void plan_workspace(const t5_handle* h, int B, int Te, int Td, char* base, Works
     return f;
   };
   w->status = (int*)take(4);          // first, so its address does not depend on the batch shape
+  w->sk_flags = (int*)take((int64_t)kSkSlices * kSkSliceInts * 4);   // per-GEMM flag slices of the stream-K tails
   w->enc_attn.clear(); w->enc_ffn.clear(); w->dec_self.clear(); w->dec_cross.clear(); w->dec_ffn.clear();
   if (encdec) {
     for (int l = 0; l < c.n_enc_layers; ++l) {
@@ -247,6 +249,7 @@ struct Ctx {
   cudaError_t err;
   const char* where;
   int64_t launches;
+  int sk_next;        // next unused flag slice
 };
 
 enum { CAT_GEMM = 0, CAT_ATTN_FWD, CAT_ATTN_BWD, CAT_NORM, CAT_GEGLU, CAT_XENT, CAT_EMBED, CAT_MISC };
@@ -292,9 +295,11 @@ struct ProfScope {
     }                                                             \
   } while (0)
 
-void gemm(Ctx& cx, const GemmArgs& g, const char* what) {
+void gemm(Ctx& cx, const GemmArgs& g0, const char* what) {
   int dt = cx.h->cfg.dtype;
   if (cx.err != cudaSuccess) return;
+  GemmArgs g = g0;
+  if (g.out_f32 && cx.sk_next < kSkSlices) g.sk_flags = cx.w->sk_flags + (cx.sk_next++) * kSkSliceInts;
   ProfScope ps(cx, CAT_GEMM, 2.0 * g.M * g.N * g.K, 1);
   if (dt == DT_BF16 && !(cx.h->cfg.flags & 1) && gemm_tc_supported(g)) {
     CK(gemm_tc(g, cx.w->status, cx.st), what);
@@ -492,6 +497,7 @@ void run_prep(Ctx& cx, const t5_batch* b) {
   Workspace& w = *cx.w;
   const t5_config& c = cx.h->cfg;
   CK(cudaMemsetAsync(w.status, 0, 4, cx.st), "memset status");
+  CK(cudaMemsetAsync(w.sk_flags, 0, (int64_t)kSkSlices * kSkSliceInts * 4, cx.st), "memset stream-K flags");
   CKL(CAT_MISC, 2, launch_prep(c.arch == 0 ? b->d_enc_tokens : nullptr, b->d_enc_segment_ids, b->d_dec_targets,
                  b->d_dec_segment_ids, cx.B, cx.Te, cx.Td, w.enc_code, w.dec_code, w.dec_in, w.W_int, w.W_f, cx.st),
      "prep");
@@ -625,7 +631,7 @@ int begin_call(t5_handle* h, const void* params, const t5_batch* b, void* ws, in
     return fail(h, T5_ERR_WORKSPACE, "workspace of %lld bytes given, %lld needed", (long long)ws_bytes,
                 (long long)w->bytes);
   cx->h = h; cx->params = params; cx->grads = nullptr; cx->st = (cudaStream_t)stream; cx->w = w;
-  cx->B = b->B; cx->Te = Te; cx->Td = b->Td; cx->err = cudaSuccess; cx->where = ""; cx->launches = 0;
+  cx->B = b->B; cx->Te = Te; cx->Td = b->Td; cx->err = cudaSuccess; cx->where = ""; cx->launches = 0; cx->sk_next = 0;
   return T5_OK;
 }
 
@@ -868,13 +874,13 @@ int t5_attention(int32_t dtype, int32_t impl, int32_t backward, int32_t B, int32
 
 int t5_gemm(int32_t dtype, int32_t impl, int32_t M, int32_t N, int32_t K, float alpha, const void* d_A, int32_t lda,
             int32_t a_kmajor, const void* d_B, int32_t ldb, int32_t b_kmajor, void* d_D, int32_t ldd,
-            int32_t out_f32, int32_t accumulate, void* stream) {
+            int32_t out_f32, int32_t accumulate, int32_t* d_sk_flags, void* stream) {
   if (!d_A || !d_B || !d_D) return T5_ERR_NULL;
   if (M < 0 || N < 0 || K < 0 || (dtype != DT_F32 && dtype != DT_BF16)) return T5_ERR_ARG;
   GemmArgs g{};
   g.M = M; g.N = N; g.K = K; g.alpha = alpha; g.A = d_A; g.lda = lda; g.a_kmajor = a_kmajor;
   g.B = d_B; g.ldb = ldb; g.b_kmajor = b_kmajor; g.D = d_D; g.ldd = ldd;
-  g.out_f32 = (dtype == DT_F32) ? 1 : out_f32; g.accumulate = accumulate;
+  g.out_f32 = (dtype == DT_F32) ? 1 : out_f32; g.accumulate = accumulate; g.sk_flags = d_sk_flags;
   cudaError_t e;
   if (impl == 0) {
     e = gemm_simt(dtype, g, (cudaStream_t)stream);

@@ -351,3 +351,26 @@ def test_gemm_tcgen05_strided_views():
     got = out.float().cpu().numpy()
     assert np.abs(got[:, 64:64 + N] - ref).max() <= 6e-3 * np.abs(ref).max()
     assert np.all(got[:, :64] == 0) and np.all(got[:, 64 + N:] == 0)
+
+
+@pytest.mark.parametrize("ak,bk", [(0, 0), (1, 1)])
+@pytest.mark.parametrize("M,N,K", [(2048, 2048, 4096), (2048, 5120, 2048), (6144, 2048, 3648), (1000, 520, 1104)])
+def test_gemm_tcgen05_stream_k_tail(ak, bk, M, N, K):
+    """float32-output GEMMs whose last wave is partial: its tiles are cut along K over all SMs
+    (one segment stores, the others add atomically); result must equal the plain schedule."""
+    rng = np.random.default_rng(M + N + K)
+    A = torch.from_numpy(rng.standard_normal((M, K)).astype(np.float32)).to(DEV).to(torch.bfloat16)
+    Bm = torch.from_numpy(rng.standard_normal((N, K)).astype(np.float32)).to(DEV).to(torch.bfloat16)
+    ref = A.double().cpu().numpy() @ Bm.double().cpu().numpy().T
+    As = A if ak else A.t().contiguous()
+    Bs = Bm if bk else Bm.t().contiguous()
+    scale = np.abs(ref).max()
+    flags = torch.zeros(160, dtype=torch.int32, device=DEV)
+    D = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
+    Bd.t5_gemm(1, M, N, K, 0.5, As, As.stride(0), ak, Bs, Bs.stride(0), bk, D, N, sk_flags=flags)
+    torch.cuda.synchronize()
+    assert np.abs(D.cpu().numpy() - 0.5 * ref).max() <= 2e-5 * scale
+    flags.zero_()
+    Bd.t5_gemm(1, M, N, K, 0.25, As, As.stride(0), ak, Bs, Bs.stride(0), bk, D, N, accumulate=True, sk_flags=flags)
+    torch.cuda.synchronize()
+    assert np.abs(D.cpu().numpy() - 0.75 * ref).max() <= 2e-5 * scale
