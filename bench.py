@@ -140,6 +140,21 @@ class OracleSample:
         return time.perf_counter() - t0
 
 
+def max_over_ranks(ms, dist=None, device=None):
+    """The job's time is the slowest rank's: all-reduce MAX of the per-rank device time (no-op on one rank)."""
+    if dist is None:
+        return float(ms)
+    import torch
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_rank_step, world, ms_total, steps):
+    """tokens/s of all ranks together (every rank runs an independent replica on its own batch)."""
+    return world * tokens_per_rank_step / (ms_total * 1e-3 / steps)
+
+
 def cpu_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -251,12 +266,7 @@ def main():
             fn()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), dist, dev)
 
     for _ in range(args.warmup):
         step()
@@ -308,7 +318,7 @@ def main():
     achieved_tf = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
 
     sec = ms * 1e-3 / args.steps
-    value = world * tokens_per_step / sec
+    value = whole_job_value(tokens_per_step, world, ms, args.steps)
     sec_e2e = ms_e2e * 1e-3 / args.steps
     out = {
         "metric": "train_tokens_per_sec", "value": value, "unit": "tokens/s", "n_gpus": world,

@@ -380,3 +380,37 @@ def test_gemm_tcgen05_stream_k_tail(ak, bk, M, N, K):
     Bd.t5_gemm(1, M, N, K, 0.25, As, As.stride(0), ak, Bs, Bs.stride(0), bk, D, N, accumulate=True, sk_flags=flags)
     torch.cuda.synchronize()
     assert np.abs(D.cpu().numpy() - 0.75 * ref).max() <= 2e-5 * scale
+
+
+# ------------------------------------------------------------------ degenerate and boundary shapes
+@pytest.mark.parametrize("Te,Td", [(1, 1), (128, 64), (129, 65), (64, 128)])
+def test_step_boundary_lengths_bf16(Te, Td):
+    """Lengths of one token, exact multiples of the 64/128 tiles, and one past them (tensor-core path, d_kv = 64)."""
+    dims = WL.model_dims("small", n_enc_layers=1, n_dec_layers=1, vocab=512, d_model=128, n_heads=2, d_ff=128,
+                         enc_len=Te, dec_len=Td, batch=3, padding=0.0)
+    batch = WL.make_batch(dims, seed=Te * 7 + Td)
+    check_step(dims, batch, "bf16", floor=True)
+
+
+def test_step_rows_without_targets_and_without_inputs():
+    """A row whose targets are all padding, and a row whose encoder input is all padding (its decoder queries see
+    no encoder key): both must contribute exactly what the oracle says (zero attention output, finite gradients)."""
+    dims = WL.model_dims("small", n_enc_layers=1, n_dec_layers=2, vocab=512, d_model=128, n_heads=2, d_ff=128,
+                         enc_len=70, dec_len=33, batch=4, padding=0.0)
+    batch = WL.make_batch(dims, seed=3)
+    batch["dec_targets"][1, :] = 0
+    batch["enc_tokens"][2, :] = 0
+    for dtype in ("f32", "bf16"):
+        check_step(dims, batch, dtype, floor=True)
+
+
+def test_max_configured_sizes_are_accepted_and_one_more_is_not():
+    dims = WL.model_dims("tiny")
+    r = Runner(dims, 2, 16, 8, "f32")
+    r.set_params(WL.make_params(PR.oracle_shapes_from_manifest(r.man), 1))
+    ok = WL.make_batch(WL.model_dims("tiny", batch=2, enc_len=16, dec_len=8))
+    r.step(ok)
+    for kw in (dict(batch=2, enc_len=17, dec_len=8), dict(batch=2, enc_len=16, dec_len=9)):
+        with pytest.raises(Bd.T5Error) as e:
+            r.step(WL.make_batch(WL.model_dims("tiny", **kw)))
+        assert e.value.code == -3
