@@ -70,7 +70,8 @@ typedef struct {
   int32_t recompute;        /* activation policy: 0 keep everything, 1 recompute cheap
                                element-wise pieces in the backward pass */
   int32_t flags;            /* debugging aids for bfloat16 mode: bit 0 = use the plain SIMT
-                               GEMM kernel, bit 1 = use the plain SIMT attention kernels.
+                               GEMM kernel, bit 1 = use the plain SIMT attention kernels,
+                               bit 2 = run the GEMMs on CTA pairs (cta_group::2).
                                In float32 mode bits 4..16 round one family of intermediates
                                to bfloat16 in place (normed activations, projections, context,
                                FFN pre-activations, gated product, logits, dlogits, residual
@@ -186,7 +187,8 @@ T5_API int t5_xent_zloss(int32_t dtype, void* d_logits, const int32_t* d_targets
 /* D[M,N] = alpha * A * B (+ D when accumulate), bf16/f32 operands, f32 accumulation.
  * a_kmajor: A is stored [M,K] (else [K,M]); b_kmajor: B is stored [N,K] (else [K,N]);
  * lda/ldb/ldd are row strides in elements.  out_f32: D is float32, else the operand
- * dtype.  impl 0 = SIMT kernel, 1 = tcgen05/TMEM/TMA kernel (bfloat16 only).
+ * dtype.  impl 0 = SIMT kernel, 1 = tcgen05/TMEM/TMA kernel (bfloat16 only), 2 = the same on
+ * CTA pairs (cta_group::2, 256 x 256 tiles) where M, N >= 256.
  * d_sk_flags: NULL, or 160 zeroed int32 that allow the tcgen05 kernel to cut the
  * tiles of a partial last wave along K over all SMs (float32 output only). */
 T5_API int t5_gemm(int32_t dtype, int32_t impl, int32_t M, int32_t N, int32_t K, float alpha,

@@ -70,6 +70,7 @@ cudaError_t gemm_simt(int dtype, const GemmArgs& g, cudaStream_t st);
 // bounded wait inside the kernel ran out.
 cudaError_t gemm_tc(const GemmArgs& g, int* d_status, cudaStream_t st);
 bool gemm_tc_supported(const GemmArgs& g);
+void gemm_tc_set_pair_mode(int on);   // 1: 256 x 256 tiles on CTA pairs (cta_group::2) where the shape allows
 
 struct AttnArgs {
   // rows of Q/O/dQ/dO are (b*Tq + i), rows of K/V/dK/dV are (b*Tk + j);

@@ -82,6 +82,73 @@ struct WorkIter {
   }
 };
 
+// Epilogue of one 128-row x BN-column accumulator tile for one warp (rows quad*32 .. +31 of the tile).
+// Each thread holds one accumulator row; going through a per-warp shared-memory tile turns the stores (and the
+// loads of the float32 addend) into 128-byte row segments instead of 32 scattered pieces.
+template <int BN>
+__device__ __forceinline__ void store_tile(const Params& p, float* tbuf, uint32_t tacc, int m0, int n0, int quad,
+                                           int lane, bool add_atomic) {
+  const int rr0 = lane >> 3, cc = (lane & 7) * 4;
+  // float32 addend (residual input, or D itself when accumulating), fetched one chunk ahead of its use
+  const float* addend = (!p.out_f32 || add_atomic) ? nullptr
+                                                    : (p.resid ? p.resid : (p.accumulate ? (const float*)p.D : nullptr));
+  const int ld_add = p.resid ? p.ldr : p.ldd;
+  float4 add_next[8];
+  auto fetch_addend = [&](int c, float4 (&dst)[8]) {
+    const int col = n0 + c * 32 + cc;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int row = m0 + quad * 32 + i * 4 + rr0;
+      dst[i] = (addend && row < p.M && col < p.N) ? *reinterpret_cast<const float4*>(addend + (int64_t)row * ld_add + col)
+                                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  fetch_addend(0, add_next);
+#pragma unroll 1
+  for (int c = 0; c < BN / 32; ++c) {
+    const int col0 = n0 + c * 32;
+    if (col0 >= p.N) break;               // uniform across the warp
+    float4 add_cur[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) add_cur[i] = add_next[i];
+    uint32_t r[32];
+    tmem_ld_32x32b_x32(tacc + c * 32, r);
+    tmem_wait_ld_dep(r);
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      *reinterpret_cast<float4*>(tbuf + lane * 36 + j * 4) =
+          make_float4(p.alpha * __uint_as_float(r[4 * j]), p.alpha * __uint_as_float(r[4 * j + 1]),
+                      p.alpha * __uint_as_float(r[4 * j + 2]), p.alpha * __uint_as_float(r[4 * j + 3]));
+    __syncwarp();
+    if (addend && c + 1 < BN / 32) fetch_addend(c + 1, add_next);     // in flight while this chunk is stored
+    const int col = col0 + cc;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int rr = i * 4 + rr0;
+      const int row = m0 + quad * 32 + rr;
+      float4 v = *reinterpret_cast<const float4*>(tbuf + rr * 36 + cc);
+      if (row < p.M && col < p.N) {        // N is a multiple of 4: a float4 never straddles the edge
+        if (add_atomic) {
+          float* d = (float*)p.D + (int64_t)row * p.ldd + col;
+          asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(d), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+                       : "memory");
+        } else if (p.out_f32) {
+          v.x += add_cur[i].x; v.y += add_cur[i].y; v.z += add_cur[i].z; v.w += add_cur[i].w;
+          *reinterpret_cast<float4*>((float*)p.D + (int64_t)row * p.ldd + col) = v;
+        } else {
+          bf16* d = (bf16*)p.D + (int64_t)row * p.ldd + col;
+          __nv_bfloat162 b0 = __floats2bfloat162_rn(v.x, v.y), b1 = __floats2bfloat162_rn(v.z, v.w);
+          uint2 o;
+          o.x = *reinterpret_cast<uint32_t*>(&b0);
+          o.y = *reinterpret_cast<uint32_t*>(&b1);
+          *reinterpret_cast<uint2*>(d) = o;
+        }
+      }
+    }
+    __syncwarp();                          // the tile is rewritten by the next chunk
+  }
+}
+
 template <int BN, int STAGES>
 struct Smem {
   static constexpr int kABytes = BM * BK * 2;
@@ -237,69 +304,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (!ok) break;
       tc_fence_after();
       const bool add_atomic = w.kind == 2;
-      const uint32_t tacc = tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16);
-      // Each thread holds one accumulator row; going through a per-warp shared-memory tile turns the stores
-      // (and the loads of the float32 addend) into 128-byte row segments instead of 32 scattered pieces.
-      float* tbuf = reinterpret_cast<float*>(smem + S::kEpiOffset) + quad * (32 * 36);
-      const int rr0 = lane >> 3, cc = (lane & 7) * 4;
-      // float32 addend (residual input, or D itself when accumulating), fetched one chunk ahead of its use
-      const float* addend = (!p.out_f32 || add_atomic) ? nullptr
-                                                        : (p.resid ? p.resid : (p.accumulate ? (const float*)p.D : nullptr));
-      const int ld_add = p.resid ? p.ldr : p.ldd;
-      float4 add_next[8];
-      auto fetch_addend = [&](int c, float4 (&dst)[8]) {
-        const int col = n0 + c * 32 + cc;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int row = m0 + quad * 32 + i * 4 + rr0;
-          dst[i] = (addend && row < p.M && col < p.N) ? *reinterpret_cast<const float4*>(addend + (int64_t)row * ld_add + col)
-                                                        : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-      };
-      fetch_addend(0, add_next);
-#pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        const int col0 = n0 + c * 32;
-        if (col0 >= p.N) break;               // uniform across the warp
-        float4 add_cur[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) add_cur[i] = add_next[i];
-        uint32_t r[32];
-        tmem_ld_32x32b_x32(tacc + c * 32, r);
-        tmem_wait_ld_dep(r);
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-          *reinterpret_cast<float4*>(tbuf + lane * 36 + j * 4) =
-              make_float4(p.alpha * __uint_as_float(r[4 * j]), p.alpha * __uint_as_float(r[4 * j + 1]),
-                          p.alpha * __uint_as_float(r[4 * j + 2]), p.alpha * __uint_as_float(r[4 * j + 3]));
-        __syncwarp();
-        if (addend && c + 1 < BN / 32) fetch_addend(c + 1, add_next);     // in flight while this chunk is stored
-        const int col = col0 + cc;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int rr = i * 4 + rr0;
-          const int row = m0 + quad * 32 + rr;
-          float4 v = *reinterpret_cast<const float4*>(tbuf + rr * 36 + cc);
-          if (row < p.M && col < p.N) {        // N is a multiple of 4: a float4 never straddles the edge
-            if (add_atomic) {
-              float* d = (float*)p.D + (int64_t)row * p.ldd + col;
-              asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(d), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
-                           : "memory");
-            } else if (p.out_f32) {
-              v.x += add_cur[i].x; v.y += add_cur[i].y; v.z += add_cur[i].z; v.w += add_cur[i].w;
-              *reinterpret_cast<float4*>((float*)p.D + (int64_t)row * p.ldd + col) = v;
-            } else {
-              bf16* d = (bf16*)p.D + (int64_t)row * p.ldd + col;
-              __nv_bfloat162 b0 = __floats2bfloat162_rn(v.x, v.y), b1 = __floats2bfloat162_rn(v.z, v.w);
-              uint2 o;
-              o.x = *reinterpret_cast<uint32_t*>(&b0);
-              o.y = *reinterpret_cast<uint32_t*>(&b1);
-              *reinterpret_cast<uint2*>(d) = o;
-            }
-          }
-        }
-        __syncwarp();                          // the tile is rewritten by the next chunk
-      }
+      store_tile<BN>(p, reinterpret_cast<float*>(smem + S::kEpiOffset) + quad * (32 * 36),
+                     tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16), m0, n0, quad, lane, add_atomic);
       if (w.kind == 1) {          // publish this warp's part of the stored tile to the adding segments
         __threadfence();
         __syncwarp();
@@ -319,6 +325,148 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   }
 }
 
+
+// ============================================================================ two-CTA variant
+// A cluster of two CTAs computes one 256 x 256 tile: CTA r loads rows [128 r, 128 r + 128) of A and of the B tile
+// into its own shared memory (plain TMA, completion counted on the leader's barrier), the leader's MMA thread issues
+// tcgen05.mma.cta_group::2 (M = 256, N = 256), each CTA's tensor memory receives its 128 rows of the result and each
+// CTA runs the epilogue of its half.  Per CTA a K slice costs 32 KB of loads instead of 48 KB, and six stages fit.
+constexpr int STAGES2 = 6;
+struct Smem2 {
+  static constexpr int kABytes = 128 * BK * 2, kBBytes = 128 * BK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kBarOffset = STAGES2 * kStageBytes;
+  static constexpr int kEpiOffset = kBarOffset + 256;
+  static constexpr int kEpiBytes = 4 * 32 * 36 * 4;
+  static constexpr int kTotal = kEpiOffset + kEpiBytes + 1024;
+};
+
+template <bool A_MN, bool B_MN>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, Params p) {
+  using S = Smem2;
+  constexpr int BN = 256;
+  extern __shared__ unsigned char smem_raw[];
+  // both CTAs of a pair must use identical offsets: the dynamic shared-memory base is the same in both
+  unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint64_t* full = (uint64_t*)(smem + S::kBarOffset);
+  uint64_t* empty = full + STAGES2;
+  uint64_t* tfull = empty + STAGES2;      // [2]
+  uint64_t* tempty = tfull + 2;           // [2]
+  uint32_t* tmem_holder = (uint32_t*)(tempty + 2);
+  volatile int* abort_flag = (volatile int*)(tmem_holder + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const int n_tiles = p.tiles_m * p.tiles_n;             // 256 x 256 tiles
+  const int k_blocks = (p.K + BK - 1) / BK;
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  constexpr uint32_t kTmemCols = 512;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES2; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 8); }   // 4 warps of each CTA
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 2) tmem_alloc_pair(tmem_holder, kTmemCols);
+  tc_fence_before();
+  cluster_sync_all();                 // barriers of both CTAs exist before anything signals them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+        const int m0 = (tile % p.tiles_m) * 256 + (int)rank * 128, n0 = (tile / p.tiles_m) * 256 + (int)rank * 128;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status, 6)) { ok = false; break; }
+          unsigned char* sa = smem + s * S::kStageBytes;
+          unsigned char* sb = sa + S::kABytes;
+          if (leader) mbar_arrive_expect_tx(&full[s], 2 * S::kStageBytes);     // both CTAs' bytes land on this barrier
+          const int k0 = kb * BK;
+          if (!A_MN) {
+            tma_load_2d_pair(sa, &map_a, k0, m0, &full[s]);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 2; ++c) tma_load_2d_pair(sa + c * 8192, &map_a, m0 + c * 64, k0, &full[s]);
+          }
+          if (!B_MN) {
+            tma_load_2d_pair(sb, &map_b, k0, n0, &full[s]);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 2; ++c) tma_load_2d_pair(sb + c * 8192, &map_b, n0 + c * 64, k0, &full[s]);
+          }
+          if (++s == STAGES2) { s = 0; ph ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && leader) {
+      constexpr uint32_t idesc = make_idesc(256, 256, A_MN, B_MN);
+      int s = 0;
+      uint32_t ph = 0;
+      int it = 0;
+      bool ok = true;
+      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++it) {
+        const int ab = it & 1;
+        const uint32_t aph = (it >> 1) & 1;
+        if (!mbar_wait(&tempty[ab], aph ^ 1, abort_flag, p.status, 7)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tacc = tmem_base + ab * BN;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(&full[s], ph, abort_flag, p.status, 8)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + s * S::kStageBytes);
+          const uint32_t sb = sa + S::kABytes;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            uint64_t da = A_MN ? make_desc(sa + k * 2048, 8192, 1024) : make_desc(sa + k * 32, 16, 1024);
+            uint64_t db = B_MN ? make_desc(sb + k * 2048, 8192, 1024) : make_desc(sb + k * 32, 16, 1024);
+            umma_bf16_pair(tacc, da, db, idesc, (kb | k) != 0);
+          }
+          umma_commit_pair(&empty[s]);            // frees the stage in both CTAs
+          if (++s == STAGES2) { s = 0; ph ^= 1; }
+        }
+        if (ok) umma_commit_pair(&tfull[ab]);     // both CTAs' epilogues may read their half
+      }
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
+    const int quad = warp & 3;
+    int it = 0;
+    bool ok = true;
+    for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++it) {
+      const int m0 = (tile % p.tiles_m) * 256 + (int)rank * 128, n0 = (tile / p.tiles_m) * 256;
+      const int ab = it & 1;
+      const uint32_t aph = (it >> 1) & 1;
+      ok = mbar_wait(&tfull[ab], aph, abort_flag, p.status, 9);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      store_tile<BN>(p, reinterpret_cast<float*>(smem + S::kEpiOffset) + quad * (32 * 36),
+                     tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16), m0, n0, quad, lane, false);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_leader(&tempty[ab]);
+    }
+  }
+
+  tc_fence_before();
+  cluster_sync_all();                 // the peer's shared memory and barriers stay alive until both are done
+  if (warp == 2) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
+  }
+}
+
 // ----------------------------------------------------------------------------- host side
 // 2-D bf16 tensor [outer, inner] (inner contiguous, row stride ld elements); box = [box_outer, 64]
 bool make_map(CUtensorMap* m, const void* base, int64_t inner, int64_t outer, int64_t ld, int box_outer) {
@@ -335,6 +483,7 @@ bool make_map(CUtensorMap* m, const void* base, int64_t inner, int64_t outer, in
 }
 
 int g_num_sms = 0;
+int g_pair_mode = 0;      // 1: use the two-CTA kernel where it applies
 
 template <int BN, int STAGES, bool A_MN, bool B_MN>
 cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& mb, int* status, cudaStream_t st) {
@@ -367,6 +516,39 @@ cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& 
   return cudaGetLastError();
 }
 
+template <bool A_MN, bool B_MN>
+cudaError_t launch2(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& mb, int* status, cudaStream_t st) {
+  static bool configured = false;
+  auto kern = gemm_tc2_kernel<A_MN, B_MN>;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem2::kTotal);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  Params p;
+  p.M = g.M; p.N = g.N; p.K = g.K; p.alpha = g.alpha; p.D = g.D; p.ldd = g.ldd; p.out_f32 = g.out_f32;
+  p.resid = g.resid; p.ldr = g.ldr; p.accumulate = g.accumulate;
+  p.tiles_m = (g.M + 255) / 256; p.tiles_n = (g.N + 255) / 256; p.status = status;
+  p.sk_full = 0; p.sk_rem = 0; p.sk_flags = nullptr;
+  int tiles = p.tiles_m * p.tiles_n;
+  int pairs = g_num_sms / 2;
+  if (tiles < pairs) pairs = tiles;
+  kern<<<2 * pairs, kThreads, Smem2::kTotal, st>>>(ma, mb, p);
+  return cudaGetLastError();
+}
+
+// 256 x 256 tiles on CTA pairs: boxes are 128 rows (K-major) or 64 x 64 (MN-major), as for BN = 128
+cudaError_t dispatch2(const GemmArgs& g, int* status, cudaStream_t st) {
+  CUtensorMap ma, mb;
+  bool ok = g.a_kmajor ? make_map(&ma, g.A, g.K, g.M, g.lda, 128) : make_map(&ma, g.A, g.M, g.K, g.lda, 64);
+  ok = ok && (g.b_kmajor ? make_map(&mb, g.B, g.K, g.N, g.ldb, 128) : make_map(&mb, g.B, g.N, g.K, g.ldb, 64));
+  if (!ok) return cudaErrorInvalidValue;
+  if (g.a_kmajor && g.b_kmajor) return launch2<false, false>(g, ma, mb, status, st);
+  if (g.a_kmajor) return launch2<false, true>(g, ma, mb, status, st);
+  if (g.b_kmajor) return launch2<true, false>(g, ma, mb, status, st);
+  return launch2<true, true>(g, ma, mb, status, st);
+}
+
 template <int BN, int STAGES>
 cudaError_t dispatch(const GemmArgs& g, int* status, cudaStream_t st) {
   CUtensorMap ma, mb;
@@ -395,6 +577,8 @@ bool gemm_tc_supported(const GemmArgs& g) {
   return tc::get_encode() != nullptr;
 }
 
+void gemm_tc_set_pair_mode(int on) { g_pair_mode = on; }
+
 cudaError_t gemm_tc(const GemmArgs& g, int* d_status, cudaStream_t st) {
   if (g_num_sms == 0) {
     int dev = 0;
@@ -403,6 +587,7 @@ cudaError_t gemm_tc(const GemmArgs& g, int* d_status, cudaStream_t st) {
     e = cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
   }
+  if (g_pair_mode == 1 && g.M >= 256 && g.N >= 256) return dispatch2(g, d_status, st);
   // wide tiles unless N is small enough that they would mostly compute padding
   if (g.N > 128) return dispatch<256, 4>(g, d_status, st);
   return dispatch<128, 6>(g, d_status, st);

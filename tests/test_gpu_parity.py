@@ -414,3 +414,27 @@ def test_max_configured_sizes_are_accepted_and_one_more_is_not():
         with pytest.raises(Bd.T5Error) as e:
             r.step(WL.make_batch(WL.model_dims("tiny", **kw)))
         assert e.value.code == -3
+
+
+@pytest.mark.parametrize("ak,bk", [(1, 1), (1, 0), (0, 0), (0, 1)])
+@pytest.mark.parametrize("M,N,K", [(256, 256, 64), (512, 768, 512), (1000, 520, 200), (3648, 2048, 2048)])
+def test_gemm_tcgen05_cta_pairs(ak, bk, M, N, K):
+    """256 x 256 tiles on CTA pairs (tcgen05.mma.cta_group::2) against the float64 product."""
+    rng = np.random.default_rng(M + N + K + 1)
+    A = torch.from_numpy(rng.standard_normal((M, K)).astype(np.float32)).to(DEV).to(torch.bfloat16)
+    Bm = torch.from_numpy(rng.standard_normal((N, K)).astype(np.float32)).to(DEV).to(torch.bfloat16)
+    ref = A.double().cpu().numpy() @ Bm.double().cpu().numpy().T
+    As = A if ak else A.t().contiguous()
+    Bs = Bm if bk else Bm.t().contiguous()
+    scale = np.abs(ref).max()
+    D = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=DEV)
+    Bd.t5_gemm(2, M, N, K, 1.0, As, As.stride(0), ak, Bs, Bs.stride(0), bk, D, N)
+    torch.cuda.synchronize()
+    got = D.float().cpu().numpy()
+    assert np.isfinite(got).all()
+    assert np.abs(got - ref).max() <= 6e-3 * scale
+    D32 = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
+    Bd.t5_gemm(2, M, N, K, 0.5, As, As.stride(0), ak, Bs, Bs.stride(0), bk, D32, N)
+    Bd.t5_gemm(2, M, N, K, 0.25, As, As.stride(0), ak, Bs, Bs.stride(0), bk, D32, N, accumulate=True)
+    torch.cuda.synchronize()
+    assert np.abs(D32.cpu().numpy() - 0.75 * ref).max() <= 2e-5 * scale
