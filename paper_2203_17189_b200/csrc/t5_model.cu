@@ -630,7 +630,7 @@ int begin_call(t5_handle* h, const void* params, const t5_batch* b, void* ws, in
   if (w->bytes > ws_bytes)
     return fail(h, T5_ERR_WORKSPACE, "workspace of %lld bytes given, %lld needed", (long long)ws_bytes,
                 (long long)w->bytes);
-  gemm_tc_set_pair_mode((h->cfg.flags >> 2) & 1);
+  gemm_tc_set_pair_mode(((h->cfg.flags >> 2) & 1) ^ 1);     // CTA pairs unless flag bit 2 says otherwise
   cx->h = h; cx->params = params; cx->grads = nullptr; cx->st = (cudaStream_t)stream; cx->w = w;
   cx->B = b->B; cx->Te = Te; cx->Td = b->Td; cx->err = cudaSuccess; cx->where = ""; cx->launches = 0; cx->sk_next = 0;
   return T5_OK;
