@@ -100,6 +100,7 @@ __global__ void rmsnorm_fwd_kernel(const float* __restrict__ X, const T* __restr
   if (row >= rows) return;
   const float* x = X + (int64_t)row * d;
   float ss = 0.f;
+#pragma unroll 4
   for (int c = lane * 4; c < d; c += 128) {
     float4 v = load4(x + c);
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
@@ -108,6 +109,7 @@ __global__ void rmsnorm_fwd_kernel(const float* __restrict__ X, const T* __restr
   float r = rsqrtf(ss / (float)d + eps);
   if (lane == 0) rstd[row] = r;
   T* y = Y + (int64_t)row * d;
+#pragma unroll 4
   for (int c = lane * 4; c < d; c += 128) {
     float4 v = load4(x + c);
     float4 gg = load4(g + c);
@@ -137,6 +139,7 @@ __global__ void rmsnorm_bwd_kernel(const TDY* __restrict__ dY, const float* __re
     const TDY* dy = dY + (int64_t)row * d;
     float r = rstd[row];
     float m = 0.f;
+#pragma unroll 4
     for (int c = lane * 4; c < d; c += 128) {
       float4 xv = load4(x + c), dv = load4(dy + c), gv = load4(g + c);
       m += dv.x * gv.x * xv.x + dv.y * gv.y * xv.y + dv.z * gv.z * xv.z + dv.w * gv.w * xv.w;
@@ -187,11 +190,20 @@ __global__ void rmsnorm_bwd_kernel(const TDY* __restrict__ dY, const float* __re
 }
 
 __global__ void colsum_kernel(const float* __restrict__ partial, int n_part, int d, float* __restrict__ out) {
-  int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= d) return;
+  // block (32, 16): 32 columns, the partial rows split over 16 groups, then a shared-memory tree
+  __shared__ float red[16][33];
+  int c = blockIdx.x * 32 + threadIdx.x;
   float s = 0.f;
-  for (int p = 0; p < n_part; ++p) s += partial[(int64_t)p * d + c];
-  out[c] = s;
+  if (c < d)
+    for (int p = threadIdx.y; p < n_part; p += 16) s += partial[(int64_t)p * d + c];
+  red[threadIdx.y][threadIdx.x] = s;
+  __syncthreads();
+  if (threadIdx.y == 0 && c < d) {
+    float t = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) t += red[i][threadIdx.x];
+    out[c] = t;
+  }
 }
 
 // ------------------------------------------------------------------ gated GELU
@@ -221,34 +233,70 @@ __device__ __forceinline__ float gelu_tanh_f(float u) {
   return 0.5f * u * (1.f + tanh_sel<FAST>(c * (u + a * u * u * u)));
 }
 
-// h [rows, 2F] = [a | b]; hg = gelu(a) * b
+// 8 consecutive elements as floats: one 16-byte access for bf16, two for float
+struct F8 { float v[8]; };
+__device__ __forceinline__ F8 load8(const float* p) {
+  float4 a = load4(p), b = load4(p + 4);
+  return {{a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w}};
+}
+__device__ __forceinline__ F8 load8(const bf16* p) {
+  uint4 u = *reinterpret_cast<const uint4*>(p);
+  F8 r;
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    r.v[2 * i] = __uint_as_float(w[i] << 16);
+    r.v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+  return r;
+}
+__device__ __forceinline__ void store8(float* p, const F8& f) {
+  store4(p, make_float4(f.v[0], f.v[1], f.v[2], f.v[3]));
+  store4(p + 4, make_float4(f.v[4], f.v[5], f.v[6], f.v[7]));
+}
+__device__ __forceinline__ void store8(bf16* p, const F8& f) {
+  uint4 u;
+  __nv_bfloat162 t;
+  t = __floats2bfloat162_rn(f.v[0], f.v[1]); u.x = *reinterpret_cast<uint32_t*>(&t);
+  t = __floats2bfloat162_rn(f.v[2], f.v[3]); u.y = *reinterpret_cast<uint32_t*>(&t);
+  t = __floats2bfloat162_rn(f.v[4], f.v[5]); u.z = *reinterpret_cast<uint32_t*>(&t);
+  t = __floats2bfloat162_rn(f.v[6], f.v[7]); u.w = *reinterpret_cast<uint32_t*>(&t);
+  *reinterpret_cast<uint4*>(p) = u;
+}
+
+// h [rows, 2F] = [a | b]; hg = gelu(a) * b     (8 elements per thread)
 template <typename T>
 __global__ void geglu_fwd_kernel(const T* __restrict__ h, T* __restrict__ hg, int rows, int F) {
   int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  int per_row = F >> 2;
+  int per_row = F >> 3;
   if (idx >= (int64_t)rows * per_row) return;
-  int r = (int)(idx / per_row), c = (int)(idx % per_row) << 2;
-  float4 a = load4(h + (int64_t)r * 2 * F + c), b = load4(h + (int64_t)r * 2 * F + F + c);
+  int r = (int)(idx / per_row), c = (int)(idx % per_row) << 3;
+  F8 a = load8(h + (int64_t)r * 2 * F + c), b = load8(h + (int64_t)r * 2 * F + F + c), o;
   constexpr bool FAST = sizeof(T) == 2;
-  store4(hg + (int64_t)r * F + c, make_float4(gelu_tanh_f<FAST>(a.x) * b.x, gelu_tanh_f<FAST>(a.y) * b.y,
-                                              gelu_tanh_f<FAST>(a.z) * b.z, gelu_tanh_f<FAST>(a.w) * b.w));
+#pragma unroll
+  for (int i = 0; i < 8; ++i) o.v[i] = gelu_tanh_f<FAST>(a.v[i]) * b.v[i];
+  store8(hg + (int64_t)r * F + c, o);
 }
 // da = dhg * b * gelu'(a); db = dhg * gelu(a)
 template <typename T>
 __global__ void geglu_bwd_kernel(const T* __restrict__ dhg, const T* __restrict__ h, T* __restrict__ dh,
                                  int rows, int F) {
   int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  int per_row = F >> 2;
+  int per_row = F >> 3;
   if (idx >= (int64_t)rows * per_row) return;
-  int r = (int)(idx / per_row), c = (int)(idx % per_row) << 2;
-  float4 a = load4(h + (int64_t)r * 2 * F + c), b = load4(h + (int64_t)r * 2 * F + F + c);
-  float4 g = load4(dhg + (int64_t)r * F + c);
+  int r = (int)(idx / per_row), c = (int)(idx % per_row) << 3;
+  F8 a = load8(h + (int64_t)r * 2 * F + c), b = load8(h + (int64_t)r * 2 * F + F + c);
+  F8 g = load8(dhg + (int64_t)r * F + c), da, db;
   constexpr bool FAST = sizeof(T) == 2;
-  float ge[4], dge[4];
-  gelu_both<FAST>(a.x, ge[0], dge[0]); gelu_both<FAST>(a.y, ge[1], dge[1]);
-  gelu_both<FAST>(a.z, ge[2], dge[2]); gelu_both<FAST>(a.w, ge[3], dge[3]);
-  store4(dh + (int64_t)r * 2 * F + c, make_float4(g.x * b.x * dge[0], g.y * b.y * dge[1], g.z * b.z * dge[2], g.w * b.w * dge[3]));
-  store4(dh + (int64_t)r * 2 * F + F + c, make_float4(g.x * ge[0], g.y * ge[1], g.z * ge[2], g.w * ge[3]));
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    float ge, dge;
+    gelu_both<FAST>(a.v[i], ge, dge);
+    da.v[i] = g.v[i] * b.v[i] * dge;
+    db.v[i] = g.v[i] * ge;
+  }
+  store8(dh + (int64_t)r * 2 * F + c, da);
+  store8(dh + (int64_t)r * 2 * F + F + c, db);
 }
 
 // ------------------------------------------------------------------ cross-entropy + z-loss
@@ -453,12 +501,12 @@ cudaError_t launch_rmsnorm_bwd(int dtype, const void* dy, int dy_f32, const floa
 #undef RB
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  colsum_kernel<<<blocks_for(d, 128), 128, 0, st>>>(partial, parts, d, dg);
+  colsum_kernel<<<blocks_for(d, 32), dim3(32, 16), 0, st>>>(partial, parts, d, dg);
   return cudaGetLastError();
 }
 
 cudaError_t launch_geglu_fwd(int dtype, const void* h, void* hg, int rows, int F, cudaStream_t st) {
-  int64_t n = (int64_t)rows * (F / 4);
+  int64_t n = (int64_t)rows * (F / 8);
   if (n == 0) return cudaSuccess;
   if (dtype == DT_F32)
     geglu_fwd_kernel<float><<<blocks_for(n, 256), 256, 0, st>>>((const float*)h, (float*)hg, rows, F);
@@ -469,7 +517,7 @@ cudaError_t launch_geglu_fwd(int dtype, const void* h, void* hg, int rows, int F
 
 cudaError_t launch_geglu_bwd(int dtype, const void* dhg, const void* h, void* dh, int rows, int F,
                              cudaStream_t st) {
-  int64_t n = (int64_t)rows * (F / 4);
+  int64_t n = (int64_t)rows * (F / 8);
   if (n == 0) return cudaSuccess;
   if (dtype == DT_F32)
     geglu_bwd_kernel<float><<<blocks_for(n, 256), 256, 0, st>>>((const float*)dhg, (const float*)h,
