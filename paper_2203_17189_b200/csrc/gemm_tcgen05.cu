@@ -82,6 +82,17 @@ struct WorkIter {
   }
 };
 
+// Tile order: groups of kGroupM tile rows are swept column by column, so that the tiles in flight at one time
+// share a few A row-blocks and a few B column-blocks (both stay in L2) instead of streaming all of A per wave.
+constexpr int kGroupM = 8;
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn) {
+  const int per_group = kGroupM * tiles_n;
+  const int g = tile / per_group, r = tile - g * per_group;
+  const int first = g * kGroupM;
+  const int gsz = min(kGroupM, tiles_m - first);
+  tm = first + r % gsz;
+  tn = r / gsz;
+}
 // Epilogue of one 128-row x BN-column accumulator tile for one warp (rows quad*32 .. +31 of the tile).
 // Each thread holds one accumulator row; going through a per-warp shared-memory tile turns the stores (and the
 // loads of the float32 addend) into 128-byte row segments instead of 32 scattered pieces.
@@ -203,7 +214,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       WorkIter wi(p, k_blocks);
       Work w;
       while (ok && wi.next(w)) {
-        const int m0 = (w.tile % p.tiles_m) * BM, n0 = (w.tile / p.tiles_m) * BN;
+        int tm, tn;
+        tile_coords(w.tile, p.tiles_m, p.tiles_n, tm, tn);
+        const int m0 = tm * BM, n0 = tn * BN;
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status, 1)) { ok = false; break; }
           unsigned char* sa = smem + s * S::kStageBytes;
@@ -282,7 +295,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     WorkIter wi(p, k_blocks);
     Work w;
     for (; ok && wi.next(w); ++it) {
-      const int m0 = (w.tile % p.tiles_m) * BM, n0 = (w.tile / p.tiles_m) * BN;
+      int tm, tn;
+        tile_coords(w.tile, p.tiles_m, p.tiles_n, tm, tn);
+        const int m0 = tm * BM, n0 = tn * BN;
       const int ab = it & 1;
       const uint32_t aph = (it >> 1) & 1;
       ok = mbar_wait(&tfull[ab], aph, abort_flag, p.status, 4);
@@ -384,7 +399,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       uint32_t ph = 0;
       bool ok = true;
       for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
-        const int m0 = (tile % p.tiles_m) * 256 + (int)rank * 128, n0 = (tile / p.tiles_m) * 256 + (int)rank * 128;
+        int tm, tn;
+        tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+        const int m0 = tm * 256 + (int)rank * 128, n0 = tn * 256 + (int)rank * 128;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status, 6)) { ok = false; break; }
           unsigned char* sa = smem + s * S::kStageBytes;
@@ -444,7 +461,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     int it = 0;
     bool ok = true;
     for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++it) {
-      const int m0 = (tile % p.tiles_m) * 256 + (int)rank * 128, n0 = (tile / p.tiles_m) * 256;
+      int tm, tn;
+      tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+      const int m0 = tm * 256 + (int)rank * 128, n0 = tn * 256;
       const int ab = it & 1;
       const uint32_t aph = (it >> 1) & 1;
       ok = mbar_wait(&tfull[ab], aph, abort_flag, p.status, 9);
