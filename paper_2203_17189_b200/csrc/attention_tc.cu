@@ -79,6 +79,25 @@ __device__ __forceinline__ int tile_code64(const int* codes, int lane) {
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
+// dst[i] = f(i) for i in [0, n) by NT threads; four loads are in flight before their stores, so the
+// set-up of a CTA costs a couple of global-memory round trips instead of one per element.
+template <int NT, typename T, typename F>
+__device__ __forceinline__ void fill_batched(T* dst, int n, int tid, F f) {
+  for (int base = tid; base < n; base += 4 * NT) {
+    T v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      int i = base + u * NT;
+      if (i < n) v[u] = f(i);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      int i = base + u * NT;
+      if (i < n) dst[i] = v[u];
+    }
+  }
+}
+
 struct Bars {
   uint64_t ld[4];      // TMA barriers (meaning per kernel)
   uint64_t mma[2];     // MMA completion barriers
@@ -131,11 +150,11 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
   }
   if (warp == 0) tmem_alloc(&bars->tmem, kTmemCols);
   const int span = p.Tq + p.Tk - 1;
-  for (int w = tid; w < tkp + 128; w += 128) {
+  fill_batched<128>(bias_s, tkp + 128, tid, [&](int w) {
     int g = w - 127 - q0 + p.Tq - 1;
-    bias_s[w] = (p.bias_delta && g >= 0 && g < span) ? p.bias_delta[(int64_t)h * span + g] * kLog2e : 0.f;
-  }
-  for (int j = tid; j < tkp; j += 128) codes_s[j] = j < p.Tk ? p.code_k[b * p.Tk + j] : 0;
+    return (p.bias_delta && g >= 0 && g < span) ? p.bias_delta[(int64_t)h * span + g] * kLog2e : 0.f;
+  });
+  fill_batched<128>(codes_s, tkp, tid, [&](int j) { return j < p.Tk ? p.code_k[b * p.Tk + j] : 0; });
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -407,12 +426,12 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
   }
   if (warp == 0) tmem_alloc(&bars->tmem, kTmemCols);
   const int span = p.Tq + p.Tk - 1;
-  for (int w = tid; w < tkp + 128; w += 256) {
+  fill_batched<256>(bias_s, tkp + 128, tid, [&](int w) {
     int g = w - 127 - q0 + p.Tq - 1;
-    bias_s[w] = (p.bias_delta && g >= 0 && g < span) ? p.bias_delta[(int64_t)h * span + g] * kLog2e : 0.f;
-  }
+    return (p.bias_delta && g >= 0 && g < span) ? p.bias_delta[(int64_t)h * span + g] * kLog2e : 0.f;
+  });
   for (int w = tid; w < 4 * wlen; w += 256) dbias_s[w] = 0.f;
-  for (int j = tid; j < tkp; j += 256) codes_s[j] = j < p.Tk ? p.code_k[b * p.Tk + j] : 0;
+  fill_batched<256>(codes_s, tkp, tid, [&](int j) { return j < p.Tk ? p.code_k[b * p.Tk + j] : 0; });
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -643,16 +662,15 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
   if (warp == 0) tmem_alloc(&bars->tmem, kTmemCols);
   const int span = p.Tq + p.Tk - 1;
   // distance of (key j = k0 + row, query i): j - i ; window index w = row - i + tqp  in [1, tqp + 127]
-  for (int w = tid; w < tqp + 128; w += 256) {
+  fill_batched<256>(bias_s, tqp + 128, tid, [&](int w) {
     int g = (w - tqp) + k0 + p.Tq - 1;
-    bias_s[w] = (p.bias_delta && g >= 0 && g < span) ? p.bias_delta[(int64_t)h * span + g] * kLog2e : 0.f;
-  }
-  for (int q = tid; q < tqp; q += 256) {
-    bool in = q < p.Tq;
-    lse_s[q] = in ? p.lse[(int64_t)(b * p.H + h) * p.Tq + q] * kLog2e : -INFINITY;
-    dl_s[q] = in ? p.delta[(int64_t)(b * p.H + h) * p.Tq + q] : 0.f;
-    codes_s[q] = in ? p.code_q[b * p.Tq + q] : 0;
-  }
+    return (p.bias_delta && g >= 0 && g < span) ? p.bias_delta[(int64_t)h * span + g] * kLog2e : 0.f;
+  });
+  fill_batched<256>(lse_s, tqp, tid, [&](int q) {
+    return q < p.Tq ? p.lse[(int64_t)(b * p.H + h) * p.Tq + q] * kLog2e : -INFINITY;
+  });
+  fill_batched<256>(dl_s, tqp, tid, [&](int q) { return q < p.Tq ? p.delta[(int64_t)(b * p.H + h) * p.Tq + q] : 0.f; });
+  fill_batched<256>(codes_s, tqp, tid, [&](int q) { return q < p.Tq ? p.code_q[b * p.Tq + q] : 0; });
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
