@@ -23,6 +23,7 @@
 #include <math.h>
 
 #include <algorithm>
+#include <type_traits>
 
 namespace {
 
@@ -46,6 +47,7 @@ struct TcParams {
   int B, H, Tq, Tk, causal;
   float scale;
   int* status;
+  int bias_far;              // see AttnArgs::bias_far
 };
 
 __device__ __forceinline__ uint64_t desc_k(uint32_t addr) { return make_desc(addr, 16, 1024); }
@@ -447,6 +449,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
   const float sc2 = p.scale * kLog2e;
   uint32_t ph_kv[3] = {0, 0, 0}, ph_m = 0;
   bool ok = true;
+  float far_pos = 0.f, far_neg = 0.f;      // dS mass of blocks wholly beyond +bias_far / -bias_far
   constexpr uint32_t idesc_s = make_idesc(128, 64, false, false);
   constexpr uint32_t idesc_dq = make_idesc(128, DK, false, true);
 
@@ -496,30 +499,55 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
     tmem_wait_ld_dep(rp);
     {
       float ds[32];
+      // four compiled variants (mask needed or not, bias or not) chosen by one warp-uniform branch, so the common
+      // unmasked case carries no mask or select instructions
+      auto compute = [&](auto fast_c, auto bias_c) {
+        constexpr bool FAST = decltype(fast_c)::value, BIAS = decltype(bias_c)::value;
 #pragma unroll
-      for (int jj = 0; jj < 32; ++jj) {
-        float sv = has_bias ? fmaf(__uint_as_float(rs[jj]), sc2, brow[c * 32 + jj]) : __uint_as_float(rs[jj]) * sc2;
-        float pr = ex2_approx(sv - lse2);
-        if (!fast) {
-          int j = k0 + c * 32 + jj;
-          int ck = codes_s[j];
-          bool valid = ck != 0 && ck == cq && (!p.causal || j <= i) && lse2 != -INFINITY;
-          pr = valid ? pr : 0.f;
+        for (int jj = 0; jj < 32; ++jj) {
+          float sv = BIAS ? fmaf(__uint_as_float(rs[jj]), sc2, brow[c * 32 + jj]) : __uint_as_float(rs[jj]) * sc2;
+          float pr = ex2_approx(sv - lse2);
+          if (!FAST) {
+            int j = k0 + c * 32 + jj;
+            int ck = codes_s[j];
+            bool valid = ck != 0 && ck == cq && (!p.causal || j <= i) && lse2 != -INFINITY;
+            pr = valid ? pr : 0.f;
+          }
+          ds[jj] = pr * (__uint_as_float(rp[jj]) - dl);
         }
-        ds[jj] = pr * (__uint_as_float(rp[jj]) - dl);
+      };
+      if (fast) {
+        if (has_bias) compute(std::true_type{}, std::true_type{}); else compute(std::true_type{}, std::false_type{});
+      } else {
+        if (has_bias) compute(std::false_type{}, std::true_type{}); else compute(std::false_type{}, std::false_type{});
       }
       if (want_db) {
-        // Diagonal sums of this warp's 32 x 32 block: at step t lane l takes column t of row (l + t) mod 32,
-        // which lies on diagonal (col - row) = -l when l + t < 32 and 32 - l otherwise.
-        float a0 = 0.f, a1 = 0.f;
+        const int kk0 = k0 + c * 32, i_lo = q0 + (quad << 5);       // this warp's 32 keys x 32 rows
+        if (p.bias_far > 0 && kk0 - (i_lo + 31) >= p.bias_far) {
+          // every (row, key) of the block is at least bias_far to the right: one bucket, plain sums
+          float t0 = 0.f, t1 = 0.f;
 #pragma unroll
-        for (int t2 = 0; t2 < 32; ++t2) {
-          float v = __shfl_sync(0xffffffffu, ds[t2], (lane + t2) & 31);
-          if (lane + t2 < 32) a0 += v; else a1 += v;
+          for (int jj = 0; jj < 32; jj += 2) { t0 += ds[jj]; t1 += ds[jj + 1]; }
+          far_pos += t0 + t1;
+        } else if (p.bias_far > 0 && i_lo - (kk0 + 31) >= p.bias_far) {
+          float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+          for (int jj = 0; jj < 32; jj += 2) { t0 += ds[jj]; t1 += ds[jj + 1]; }
+          far_neg += t0 + t1;
+        } else {
+          // Diagonal sums of the block: at step t lane l takes column t of row (l + t) mod 32, which lies on
+          // diagonal (col - row) = -l when l + t < 32 and 32 - l otherwise.
+          float tot = 0.f, a1 = 0.f;
+#pragma unroll
+          for (int t2 = 0; t2 < 32; ++t2) {
+            float v = __shfl_sync(0xffffffffu, ds[t2], (lane + t2) & 31);
+            tot += v;
+            a1 += (lane >= 32 - t2) ? v : 0.f;
+          }
+          // window entry (col - row + 31); the two column halves of a row quarter overlap there: atomics
+          atomicAdd(&dbwin[c * 32 + 31 - lane], tot - a1);
+          atomicAdd(&dbwin[c * 32 + 63 - lane], a1);
         }
-        // window entry (col - row + 31); the two column halves of a row quarter overlap there: atomics
-        atomicAdd(&dbwin[c * 32 + 31 - lane], a0);
-        atomicAdd(&dbwin[c * 32 + 63 - lane], a1);
       }
 #pragma unroll
       for (int q8 = 0; q8 < 4; ++q8) {
@@ -574,6 +602,18 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
   }
   tc_fence_before();
   __syncthreads();
+  if (ok && want_db && p.bias_far > 0) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      far_pos += __shfl_xor_sync(0xffffffffu, far_pos, o);
+      far_neg += __shfl_xor_sync(0xffffffffu, far_neg, o);
+    }
+    if ((tid & 31) == 0) {
+      const int gp = p.bias_far + p.Tq - 1, gn = -p.bias_far + p.Tq - 1;
+      if (far_pos != 0.f && gp < span) atomicAdd(&p.dbias_delta[(int64_t)h * span + gp], far_pos);
+      if (far_neg != 0.f && gn >= 0) atomicAdd(&p.dbias_delta[(int64_t)h * span + gn], far_neg);
+    }
+  }
   if (ok && want_db) {
     // CTA-level index (key - row + 127) = warp-level index + 96 - 32 * warp
     for (int w = tid; w < tkp + 128; w += 256) {
@@ -732,26 +772,34 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
     tmem_wait_ld_dep(rp);
     {
       float pt[32], ds[32];
+      auto compute = [&](auto fast_c, auto bias_c) {
+        constexpr bool FAST = decltype(fast_c)::value, BIAS = decltype(bias_c)::value;
 #pragma unroll
-      for (int i4 = 0; i4 < 8; ++i4) {
-        const float4 l4 = *reinterpret_cast<const float4*>(lse_s + qb + c * 32 + i4 * 4);
-        const float4 d4 = *reinterpret_cast<const float4*>(dl_s + qb + c * 32 + i4 * 4);
+        for (int i4 = 0; i4 < 8; ++i4) {
+          const float4 l4 = *reinterpret_cast<const float4*>(lse_s + qb + c * 32 + i4 * 4);
+          const float4 d4 = *reinterpret_cast<const float4*>(dl_s + qb + c * 32 + i4 * 4);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int ii = i4 * 4 + e;
-          const float lse2 = e == 0 ? l4.x : e == 1 ? l4.y : e == 2 ? l4.z : l4.w;
-          const float dlq = e == 0 ? d4.x : e == 1 ? d4.y : e == 2 ? d4.z : d4.w;
-          float sv = has_bias ? fmaf(__uint_as_float(rs[ii]), sc2, brow[-(c * 32 + ii)]) : __uint_as_float(rs[ii]) * sc2;
-          float pr = ex2_approx(sv - lse2);
-          if (!fast) {
-            int q = qb + c * 32 + ii;
-            int cq = codes_s[q];
-            bool valid = ck != 0 && ck == cq && (!p.causal || j <= q) && lse2 != -INFINITY;
-            pr = valid ? pr : 0.f;
+          for (int e = 0; e < 4; ++e) {
+            const int ii = i4 * 4 + e;
+            const float lse2 = e == 0 ? l4.x : e == 1 ? l4.y : e == 2 ? l4.z : l4.w;
+            const float dlq = e == 0 ? d4.x : e == 1 ? d4.y : e == 2 ? d4.z : d4.w;
+            float sv = BIAS ? fmaf(__uint_as_float(rs[ii]), sc2, brow[-(c * 32 + ii)]) : __uint_as_float(rs[ii]) * sc2;
+            float pr = ex2_approx(sv - lse2);
+            if (!FAST) {
+              int q = qb + c * 32 + ii;
+              int cq = codes_s[q];
+              bool valid = ck != 0 && ck == cq && (!p.causal || j <= q) && lse2 != -INFINITY;
+              pr = valid ? pr : 0.f;
+            }
+            pt[ii] = pr;
+            ds[ii] = pr * (__uint_as_float(rp[ii]) - dlq);
           }
-          pt[ii] = pr;
-          ds[ii] = pr * (__uint_as_float(rp[ii]) - dlq);
         }
+      };
+      if (fast) {
+        if (has_bias) compute(std::true_type{}, std::true_type{}); else compute(std::true_type{}, std::false_type{});
+      } else {
+        if (has_bias) compute(std::false_type{}, std::true_type{}); else compute(std::false_type{}, std::false_type{});
       }
 #pragma unroll
       for (int q8 = 0; q8 < 4; ++q8) {
@@ -879,6 +927,7 @@ bool make_map3(CUtensorMap* m, const void* base, int cols, int T, int B, int ld,
 TcParams base_params(const AttnArgs& a, int* status) {
   TcParams p{};
   p.lse = a.lse; p.delta = a.delta; p.code_q = a.code_q; p.code_k = a.code_k; p.bias_delta = a.bias_delta;
+  p.bias_far = a.bias_far;
   p.dbias_delta = a.dbias_delta; p.B = a.B; p.H = a.H; p.Tq = a.Tq; p.Tk = a.Tk; p.causal = a.causal;
   p.scale = a.scale; p.status = status;
   return p;

@@ -93,6 +93,9 @@ struct AttnArgs {
   void *dQ, *dK, *dV; int lddq, lddk, lddv;
   float* delta;             // [B,H,Tq] scratch: sum_d dO*O
   float* dbias_delta;       // [H, Tq+Tk-1] float32, accumulated (+=), or NULL
+  int bias_far;             // 0, or a distance F such that the bias is constant for (j - i) >= F and constant for
+                            // (j - i) <= -F (the saturated buckets): the backward may then add the whole dS mass
+                            // of such regions to the entries at +F / -F instead of to each distance
 };
 cudaError_t attn_fwd_simt(int dtype, const AttnArgs& a, cudaStream_t st);
 cudaError_t attn_bwd_simt(int dtype, const AttnArgs& a, cudaStream_t st);

@@ -347,7 +347,11 @@ void proj_wgrad(Ctx& cx, const void* dY, int lddy, const void* X, int ldx, int64
   gemm(cx, g, what);
 }
 
+// |key - query| from which the bucket no longer changes (the top bucket of that direction)
+int saturation_distance(const BucketSpec& s) { return s.n_thr > 0 ? s.thr[s.n_thr - 1] : s.me; }
+
 struct AttnGeom {
+  int far;           // distance from which the relative-position bucket is saturated (0: no bias)
   int Tq, Tk;
   int64_t Nq, Nk;
   const int *code_q, *code_k;
@@ -413,7 +417,7 @@ void attn_backward(Ctx& cx, const AttnP& p, const AttnWs& a, float* dX, void* dX
   dbg_round(cx, w.dctx, (int64_t)Nq * I, RB_DCTX);
   AttnArgs t;
   attn_args(cx, a, gm, cross, &t);
-  t.dO = w.dctx; t.lddo = I; t.delta = w.delta; t.dbias_delta = gm.dbias;
+  t.dO = w.dctx; t.lddo = I; t.delta = w.delta; t.dbias_delta = gm.dbias; t.bias_far = gm.far;
   if (cross) {
     t.dQ = w.dqkv; t.lddq = I;
     t.dK = w.dkv; t.dV = eoff(cx.h, w.dkv, I); t.lddk = t.lddv = 2 * I;
@@ -478,18 +482,21 @@ AttnGeom enc_geom(Ctx& cx) {
   AttnGeom g;
   g.Tq = g.Tk = cx.Te; g.Nq = g.Nk = (int64_t)cx.B * cx.Te;
   g.code_q = g.code_k = cx.w->enc_code; g.causal = 0; g.bias = cx.w->bias_enc; g.dbias = cx.w->dbias_enc;
+  g.far = saturation_distance(cx.h->spec_enc);
   return g;
 }
 AttnGeom self_geom(Ctx& cx) {
   AttnGeom g;
   g.Tq = g.Tk = cx.Td; g.Nq = g.Nk = (int64_t)cx.B * cx.Td;
   g.code_q = g.code_k = cx.w->dec_code; g.causal = 1; g.bias = cx.w->bias_dec; g.dbias = cx.w->dbias_dec;
+  g.far = saturation_distance(cx.h->spec_dec);
   return g;
 }
 AttnGeom cross_geom(Ctx& cx) {
   AttnGeom g;
   g.Tq = cx.Td; g.Tk = cx.Te; g.Nq = (int64_t)cx.B * cx.Td; g.Nk = (int64_t)cx.B * cx.Te;
   g.code_q = cx.w->dec_code; g.code_k = cx.w->enc_code; g.causal = 0; g.bias = nullptr; g.dbias = nullptr;
+  g.far = 0;
   return g;
 }
 
