@@ -62,6 +62,7 @@ struct GemmArgs {
   void* D; int ldd; int out_f32;          // D[M,N]; float32 or operand dtype
   const float* resid; int ldr;            // optional float32 addend (D may alias it)
   int accumulate;                         // D += (float32 output only)
+  int pair;                               // 1: 256 x 256 tiles on CTA pairs (cta_group::2) where M, N >= 256
   int* sk_flags;                          // optional: >= 160 zeroed ints; lets the tcgen05 kernel split the
                                           // tiles of a partial last wave along K over all SMs (float32 output)
 };
@@ -70,7 +71,6 @@ cudaError_t gemm_simt(int dtype, const GemmArgs& g, cudaStream_t st);
 // bounded wait inside the kernel ran out.
 cudaError_t gemm_tc(const GemmArgs& g, int* d_status, cudaStream_t st);
 bool gemm_tc_supported(const GemmArgs& g);
-void gemm_tc_set_pair_mode(int on);   // 1: 256 x 256 tiles on CTA pairs (cta_group::2) where the shape allows
 
 struct AttnArgs {
   // rows of Q/O/dQ/dO are (b*Tq + i), rows of K/V/dK/dV are (b*Tk + j);

@@ -501,18 +501,32 @@ bool make_map(CUtensorMap* m, const void* base, int64_t inner, int64_t outer, in
   return r == CUDA_SUCCESS;
 }
 
+// SM count of the current device (cached per device ordinal)
 int g_num_sms = 0;
-int g_pair_mode = 0;      // 1: use the two-CTA kernel where it applies
+int num_sms_of_current_device() {
+  static int cache[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  if (cache[dev] == 0) cudaDeviceGetAttribute(&cache[dev], cudaDevAttrMultiProcessorCount, dev);
+  return cache[dev];
+}
+// cudaFuncSetAttribute has to be repeated on every device that runs the kernel
+bool first_use_on_device(bool (&seen)[64]) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
+  bool first = !seen[dev];
+  seen[dev] = true;
+  return first;
+}
 
 template <int BN, int STAGES, bool A_MN, bool B_MN>
 cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& mb, int* status, cudaStream_t st) {
   using S = Smem<BN, STAGES>;
-  static bool configured = false;
+  static bool configured[64] = {false};
   auto kern = gemm_tc_kernel<BN, STAGES, A_MN, B_MN>;
-  if (!configured) {
+  if (first_use_on_device(configured)) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal);
     if (e != cudaSuccess) return e;
-    configured = true;
   }
   Params p;
   p.M = g.M; p.N = g.N; p.K = g.K; p.alpha = g.alpha; p.D = g.D; p.ldd = g.ldd; p.out_f32 = g.out_f32;
@@ -537,12 +551,11 @@ cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& 
 
 template <bool A_MN, bool B_MN>
 cudaError_t launch2(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& mb, int* status, cudaStream_t st) {
-  static bool configured = false;
+  static bool configured[64] = {false};
   auto kern = gemm_tc2_kernel<A_MN, B_MN>;
-  if (!configured) {
+  if (first_use_on_device(configured)) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem2::kTotal);
     if (e != cudaSuccess) return e;
-    configured = true;
   }
   Params p;
   p.M = g.M; p.N = g.N; p.K = g.K; p.alpha = g.alpha; p.D = g.D; p.ldd = g.ldd; p.out_f32 = g.out_f32;
@@ -596,17 +609,10 @@ bool gemm_tc_supported(const GemmArgs& g) {
   return tc::get_encode() != nullptr;
 }
 
-void gemm_tc_set_pair_mode(int on) { g_pair_mode = on; }
-
 cudaError_t gemm_tc(const GemmArgs& g, int* d_status, cudaStream_t st) {
-  if (g_num_sms == 0) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    e = cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return e;
-  }
-  if (g_pair_mode == 1 && g.M >= 256 && g.N >= 256) return dispatch2(g, d_status, st);
+  g_num_sms = num_sms_of_current_device();
+  if (g_num_sms <= 0) return cudaErrorInvalidDevice;
+  if (g.pair && g.M >= 256 && g.N >= 256) return dispatch2(g, d_status, st);
   // wide tiles unless N is small enough that they would mostly compute padding
   if (g.N > 128) return dispatch<256, 4>(g, d_status, st);
   return dispatch<128, 6>(g, d_status, st);

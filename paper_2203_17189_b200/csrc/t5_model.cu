@@ -299,6 +299,7 @@ void gemm(Ctx& cx, const GemmArgs& g0, const char* what) {
   int dt = cx.h->cfg.dtype;
   if (cx.err != cudaSuccess) return;
   GemmArgs g = g0;
+  g.pair = ((cx.h->cfg.flags >> 2) & 1) ^ 1;      // CTA pairs unless flag bit 2 says otherwise
   if (g.out_f32 && cx.sk_next < kSkSlices) g.sk_flags = cx.w->sk_flags + (cx.sk_next++) * kSkSliceInts;
   ProfScope ps(cx, CAT_GEMM, 2.0 * g.M * g.N * g.K, 1);
   if (dt == DT_BF16 && !(cx.h->cfg.flags & 1) && gemm_tc_supported(g)) {
@@ -637,7 +638,6 @@ int begin_call(t5_handle* h, const void* params, const t5_batch* b, void* ws, in
   if (w->bytes > ws_bytes)
     return fail(h, T5_ERR_WORKSPACE, "workspace of %lld bytes given, %lld needed", (long long)ws_bytes,
                 (long long)w->bytes);
-  gemm_tc_set_pair_mode(((h->cfg.flags >> 2) & 1) ^ 1);     // CTA pairs unless flag bit 2 says otherwise
   cx->h = h; cx->params = params; cx->grads = nullptr; cx->st = (cudaStream_t)stream; cx->w = w;
   cx->B = b->B; cx->Te = Te; cx->Td = b->Td; cx->err = cudaSuccess; cx->where = ""; cx->launches = 0; cx->sk_next = 0;
   return T5_OK;
@@ -894,9 +894,8 @@ int t5_gemm(int32_t dtype, int32_t impl, int32_t M, int32_t N, int32_t K, float 
     e = gemm_simt(dtype, g, (cudaStream_t)stream);
   } else {
     if (dtype != DT_BF16 || !gemm_tc_supported(g)) return T5_ERR_ARG;
-    gemm_tc_set_pair_mode(impl == 2);
+    g.pair = impl == 2;
     e = gemm_tc(g, nullptr, (cudaStream_t)stream);
-    gemm_tc_set_pair_mode(0);
   }
   return e == cudaSuccess ? T5_OK : T5_ERR_CUDA;
 }

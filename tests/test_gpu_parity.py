@@ -438,3 +438,37 @@ def test_gemm_tcgen05_cta_pairs(ak, bk, M, N, K):
     Bd.t5_gemm(2, M, N, K, 0.25, As, As.stride(0), ak, Bs, Bs.stride(0), bk, D32, N, accumulate=True)
     torch.cuda.synchronize()
     assert np.abs(D32.cpu().numpy() - 0.75 * ref).max() <= 2e-5 * scale
+
+
+def test_encode_and_decode_logits_bf16_tensor_core_path():
+    """The inference calls on the tensor-core path (d_kv = 64, bfloat16): encoder output and teacher-forced logits
+    against the oracle, and against what the training step computes for the same batch (same loss)."""
+    dims = WL.model_dims("small", n_enc_layers=2, n_dec_layers=2, vocab=1024, d_model=256, n_heads=4, d_ff=512,
+                         enc_len=150, dec_len=70, batch=3, padding=0.15)
+    batch = WL.make_batch(dims, seed=21)
+    B, Te, Td, d, V = 3, 150, 70, 256, 1024
+    r = Runner(dims, B, Te, Td, "bf16")
+    named = r.set_params(WL.make_params(PR.oracle_shapes_from_manifest(r.man), 4, stddev=0.02, scale_jitter=0.05))
+    dev_batch = {k: to_dev(v) for k, v in batch.items()}
+    enc_out = torch.empty(B, Te, d, dtype=torch.bfloat16, device=DEV)
+    logits = torch.empty(B, Td, V, dtype=torch.bfloat16, device=DEV)
+    r.h.t5_encode(r.params, dev_batch, enc_out, r.ws)
+    r.h.t5_decode_logits(r.params, dev_batch, enc_out, logits, r.ws)
+    torch.cuda.synchronize()
+    r.h.t5_device_status(r.ws)
+    ocfg = oracle_cfg(dims)
+    oe = O.t5_encode(ocfg, named, batch["enc_tokens"], None)
+    ol = O.t5_decode_logits(ocfg, named, oe, batch["enc_tokens"], None, batch["dec_targets"], None)
+    ve, vd = batch["enc_tokens"] != 0, batch["dec_targets"] != 0
+    ge, gl = enc_out.float().cpu().numpy(), logits.float().cpu().numpy()
+    assert np.isfinite(ge[ve]).all() and np.isfinite(gl[vd]).all()
+    assert np.abs(ge - oe)[ve].max() <= 2e-2 * np.abs(oe).max()
+    assert np.abs(gl - ol)[vd].max() <= 2e-2 * np.abs(ol).max()
+    # the loss of the training call on the same batch equals the loss computed from these logits
+    loss4, _ = r.step(batch)
+    lg = gl.astype(np.float64)
+    lse = np.log(np.exp(lg - lg.max(-1, keepdims=True)).sum(-1)) + lg.max(-1)
+    tgt = batch["dec_targets"]
+    nll = lse - np.take_along_axis(lg, tgt[..., None].astype(np.int64), -1)[..., 0]
+    want = ((nll + 1e-4 * lse ** 2) * vd).sum() / vd.sum()
+    assert abs(loss4[0] - want) <= 1e-3 * want
