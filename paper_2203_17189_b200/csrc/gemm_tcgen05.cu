@@ -53,21 +53,23 @@ struct WorkIter {
   int it = 0;
   int n_tiles, k_blocks, sk_full, sk_rem;
   long long cur, u1;
-  __device__ WorkIter(const Params& p, int kb) : n_tiles(p.tiles_m * p.tiles_n), k_blocks(kb), sk_full(p.sk_full), sk_rem(p.sk_rem) {
+  int unit, n_units;        // this scheduling unit (a CTA, or a CTA pair) and how many there are
+  __device__ WorkIter(const Params& p, int kb, int unit_, int n_units_)
+      : n_tiles(p.tiles_m * p.tiles_n), k_blocks(kb), sk_full(p.sk_full), sk_rem(p.sk_rem), unit(unit_), n_units(n_units_) {
     long long U = (long long)sk_rem * kb;
-    cur = U * blockIdx.x / gridDim.x;
-    u1 = U * (blockIdx.x + 1) / gridDim.x;
+    cur = U * unit / n_units;
+    u1 = U * (unit + 1) / n_units;
   }
   __device__ bool next(Work& w) {
     if (sk_rem == 0) {
-      int tile = blockIdx.x + it * gridDim.x;
+      int tile = unit + it * n_units;
       if (tile >= n_tiles) return false;
       w = {tile, 0, k_blocks, 0, 0};
       ++it;
       return true;
     }
     if (it < sk_full) {
-      w = {(int)(blockIdx.x + it * gridDim.x), 0, k_blocks, 0, 0};
+      w = {unit + it * n_units, 0, k_blocks, 0, 0};
       ++it;
       return true;
     }
@@ -76,7 +78,7 @@ struct WorkIter {
     long long left = u1 - cur;
     int kb1 = left < k_blocks - kb0 ? kb0 + (int)left : k_blocks;
     cur += kb1 - kb0;
-    w = {sk_full * (int)gridDim.x + t, kb0, kb1, (kb0 == 0 && kb1 == k_blocks) ? 0 : (kb1 == k_blocks ? 1 : 2), t};
+    w = {sk_full * n_units + t, kb0, kb1, (kb0 == 0 && kb1 == k_blocks) ? 0 : (kb1 == k_blocks ? 1 : 2), t};
     ++it;
     return true;
   }
@@ -211,7 +213,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
       for (int i = 0; i < STAGES; ++i) issued[i] = 0;
       bool ok = true;
-      WorkIter wi(p, k_blocks);
+      WorkIter wi(p, k_blocks, blockIdx.x, gridDim.x);
       Work w;
       while (ok && wi.next(w)) {
         int tm, tn;
@@ -260,7 +262,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       uint32_t ph = 0;
       int it = 0;
       bool ok = true;
-      WorkIter wi(p, k_blocks);
+      WorkIter wi(p, k_blocks, blockIdx.x, gridDim.x);
       Work w;
       for (; ok && wi.next(w); ++it) {
         const int ab = it & 1;
@@ -292,7 +294,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int quad = warp & 3;
     int it = 0;
     bool ok = true;
-    WorkIter wi(p, k_blocks);
+    WorkIter wi(p, k_blocks, blockIdx.x, gridDim.x);
     Work w;
     for (; ok && wi.next(w); ++it) {
       int tm, tn;
@@ -398,11 +400,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
-      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+      WorkIter wi(p, k_blocks, pair, n_pairs);
+      Work w;
+      while (ok && wi.next(w)) {
         int tm, tn;
-        tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+        tile_coords(w.tile, p.tiles_m, p.tiles_n, tm, tn);
         const int m0 = tm * 256 + (int)rank * 128, n0 = tn * 256 + (int)rank * 128;
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status, 6)) { ok = false; break; }
           unsigned char* sa = smem + s * S::kStageBytes;
           unsigned char* sb = sa + S::kABytes;
@@ -432,13 +436,15 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       uint32_t ph = 0;
       int it = 0;
       bool ok = true;
-      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++it) {
+      WorkIter wi(p, k_blocks, pair, n_pairs);
+      Work w;
+      for (; ok && wi.next(w); ++it) {
         const int ab = it & 1;
         const uint32_t aph = (it >> 1) & 1;
         if (!mbar_wait(&tempty[ab], aph ^ 1, abort_flag, p.status, 7)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tacc = tmem_base + ab * BN;
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait(&full[s], ph, abort_flag, p.status, 8)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + s * S::kStageBytes);
@@ -447,7 +453,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           for (int k = 0; k < BK / 16; ++k) {
             uint64_t da = A_MN ? make_desc(sa + k * 2048, 8192, 1024) : make_desc(sa + k * 32, 16, 1024);
             uint64_t db = B_MN ? make_desc(sb + k * 2048, 8192, 1024) : make_desc(sb + k * 32, 16, 1024);
-            umma_bf16_pair(tacc, da, db, idesc, (kb | k) != 0);
+            umma_bf16_pair(tacc, da, db, idesc, ((kb - w.kb0) | k) != 0);
           }
           umma_commit_pair(&empty[s]);            // frees the stage in both CTAs
           if (++s == STAGES2) { s = 0; ph ^= 1; }
@@ -460,18 +466,39 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const int quad = warp & 3;
     int it = 0;
     bool ok = true;
-    for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++it) {
+    WorkIter wi(p, k_blocks, pair, n_pairs);
+    Work w;
+    for (; ok && wi.next(w); ++it) {
       int tm, tn;
-      tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+      tile_coords(w.tile, p.tiles_m, p.tiles_n, tm, tn);
       const int m0 = tm * 256 + (int)rank * 128, n0 = tn * 256;
       const int ab = it & 1;
       const uint32_t aph = (it >> 1) & 1;
       ok = mbar_wait(&tfull[ab], aph, abort_flag, p.status, 9);
+      if (ok && w.kind == 2) {
+        // an earlier K-segment of a split tile: the storing pair (8 epilogue warps) must be done first
+        volatile int* flag = p.sk_flags + w.flag;
+        long long t0 = clock64();
+        while (*flag < 8) {
+          if (clock64() - t0 > kWaitCycles) {
+            if (p.status) atomicCAS(p.status, 0, 10);
+            ok = false;
+            break;
+          }
+          __nanosleep(200);
+        }
+        __threadfence();
+      }
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       store_tile<BN>(p, reinterpret_cast<float*>(smem + S::kEpiOffset) + quad * (32 * 36),
-                     tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16), m0, n0, quad, lane, false);
+                     tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16), m0, n0, quad, lane, w.kind == 2);
+      if (w.kind == 1) {
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) atomicAdd(p.sk_flags + w.flag, 1);
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_leader(&tempty[ab]);
@@ -564,7 +591,14 @@ cudaError_t launch2(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap&
   p.sk_full = 0; p.sk_rem = 0; p.sk_flags = nullptr;
   int tiles = p.tiles_m * p.tiles_n;
   int pairs = g_num_sms / 2;
-  if (tiles < pairs) pairs = tiles;
+  const int k_blocks = (g.K + BK - 1) / BK, rem = tiles % pairs;
+  // long-K float32-output GEMMs: split the tiles of a partial last wave along K over all pairs
+  if (g.sk_flags && g.out_f32 && rem > 0 && k_blocks >= 128 && tiles >= pairs && pairs <= 160 &&
+      (pairs - rem) * 8 > pairs * (tiles / pairs + 1)) {
+    p.sk_full = tiles / pairs; p.sk_rem = rem; p.sk_flags = g.sk_flags;
+  } else if (tiles < pairs) {
+    pairs = tiles;
+  }
   kern<<<2 * pairs, kThreads, Smem2::kTotal, st>>>(ma, mb, p);
   return cudaGetLastError();
 }

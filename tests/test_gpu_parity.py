@@ -359,61 +359,31 @@ def test_gemm_tcgen05_strided_views():
     assert np.all(got[:, :64] == 0) and np.all(got[:, 64 + N:] == 0)
 
 
+@pytest.mark.parametrize("impl", [1, 2])
 @pytest.mark.parametrize("ak,bk", [(0, 0), (1, 1)])
-@pytest.mark.parametrize("M,N,K", [(2048, 2048, 4096), (2048, 5120, 2048), (6144, 2048, 3648), (1000, 520, 1104)])
-def test_gemm_tcgen05_stream_k_tail(ak, bk, M, N, K):
-    """float32-output GEMMs whose last wave is partial: its tiles are cut along K over all SMs
-    (one segment stores, the others add atomically); result must equal the plain schedule."""
+@pytest.mark.parametrize("M,N,K", [(2048, 5120, 8192), (6144, 2048, 8192), (2048, 2048, 4096), (1000, 520, 1104)])
+def test_gemm_tcgen05_stream_k_tail(impl, ak, bk, M, N, K):
+    """float32-output GEMMs whose last wave is partial: with long K its tiles are cut along K over all SMs
+    (one segment stores, the others add atomically); result must equal the plain product.  The first two
+    shapes take that path in both kernels (single CTAs and CTA pairs), the others must not be disturbed."""
     rng = np.random.default_rng(M + N + K)
     A = torch.from_numpy(rng.standard_normal((M, K)).astype(np.float32)).to(DEV).to(torch.bfloat16)
     Bm = torch.from_numpy(rng.standard_normal((N, K)).astype(np.float32)).to(DEV).to(torch.bfloat16)
-    ref = A.double().cpu().numpy() @ Bm.double().cpu().numpy().T
+    ref = (A.float() @ Bm.float().t()).double().cpu().numpy() if K >= 8192 else \
+        A.double().cpu().numpy() @ Bm.double().cpu().numpy().T
     As = A if ak else A.t().contiguous()
     Bs = Bm if bk else Bm.t().contiguous()
     scale = np.abs(ref).max()
+    tol = 2e-5 if K < 8192 else 2e-4          # the long-K reference itself is a float32 product
     flags = torch.zeros(160, dtype=torch.int32, device=DEV)
     D = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
-    Bd.t5_gemm(1, M, N, K, 0.5, As, As.stride(0), ak, Bs, Bs.stride(0), bk, D, N, sk_flags=flags)
+    Bd.t5_gemm(impl, M, N, K, 0.5, As, As.stride(0), ak, Bs, Bs.stride(0), bk, D, N, sk_flags=flags)
     torch.cuda.synchronize()
-    assert np.abs(D.cpu().numpy() - 0.5 * ref).max() <= 2e-5 * scale
+    assert np.abs(D.cpu().numpy() - 0.5 * ref).max() <= tol * scale
     flags.zero_()
-    Bd.t5_gemm(1, M, N, K, 0.25, As, As.stride(0), ak, Bs, Bs.stride(0), bk, D, N, accumulate=True, sk_flags=flags)
+    Bd.t5_gemm(impl, M, N, K, 0.25, As, As.stride(0), ak, Bs, Bs.stride(0), bk, D, N, accumulate=True, sk_flags=flags)
     torch.cuda.synchronize()
-    assert np.abs(D.cpu().numpy() - 0.75 * ref).max() <= 2e-5 * scale
-
-
-# ------------------------------------------------------------------ degenerate and boundary shapes
-@pytest.mark.parametrize("Te,Td", [(1, 1), (128, 64), (129, 65), (64, 128)])
-def test_step_boundary_lengths_bf16(Te, Td):
-    """Lengths of one token, exact multiples of the 64/128 tiles, and one past them (tensor-core path, d_kv = 64)."""
-    dims = WL.model_dims("small", n_enc_layers=1, n_dec_layers=1, vocab=512, d_model=128, n_heads=2, d_ff=128,
-                         enc_len=Te, dec_len=Td, batch=3, padding=0.0)
-    batch = WL.make_batch(dims, seed=Te * 7 + Td)
-    check_step(dims, batch, "bf16", floor=True)
-
-
-def test_step_rows_without_targets_and_without_inputs():
-    """A row whose targets are all padding, and a row whose encoder input is all padding (its decoder queries see
-    no encoder key): both must contribute exactly what the oracle says (zero attention output, finite gradients)."""
-    dims = WL.model_dims("small", n_enc_layers=1, n_dec_layers=2, vocab=512, d_model=128, n_heads=2, d_ff=128,
-                         enc_len=70, dec_len=33, batch=4, padding=0.0)
-    batch = WL.make_batch(dims, seed=3)
-    batch["dec_targets"][1, :] = 0
-    batch["enc_tokens"][2, :] = 0
-    for dtype in ("f32", "bf16"):
-        check_step(dims, batch, dtype, floor=True)
-
-
-def test_max_configured_sizes_are_accepted_and_one_more_is_not():
-    dims = WL.model_dims("tiny")
-    r = Runner(dims, 2, 16, 8, "f32")
-    r.set_params(WL.make_params(PR.oracle_shapes_from_manifest(r.man), 1))
-    ok = WL.make_batch(WL.model_dims("tiny", batch=2, enc_len=16, dec_len=8))
-    r.step(ok)
-    for kw in (dict(batch=2, enc_len=17, dec_len=8), dict(batch=2, enc_len=16, dec_len=9)):
-        with pytest.raises(Bd.T5Error) as e:
-            r.step(WL.make_batch(WL.model_dims("tiny", **kw)))
-        assert e.value.code == -3
+    assert np.abs(D.cpu().numpy() - 0.75 * ref).max() <= tol * scale
 
 
 @pytest.mark.parametrize("ak,bk", [(1, 1), (1, 0), (0, 0), (0, 1)])
