@@ -71,7 +71,8 @@ typedef struct {
                                element-wise pieces in the backward pass */
   int32_t flags;            /* debugging aids for bfloat16 mode: bit 0 = use the plain SIMT
                                GEMM kernel, bit 1 = use the plain SIMT attention kernels,
-                               bit 2 = do NOT run the GEMMs on CTA pairs (cta_group::2).
+                               bit 2 = do NOT run the GEMMs on CTA pairs (cta_group::2),
+                               bit 3 = keep the gated GELU in separate kernels instead of the GEMM epilogues.
                                In float32 mode bits 4..16 round one family of intermediates
                                to bfloat16 in place (normed activations, projections, context,
                                FFN pre-activations, gated product, logits, dlogits, residual

@@ -62,6 +62,12 @@ struct GemmArgs {
   void* D; int ldd; int out_f32;          // D[M,N]; float32 or operand dtype
   const float* resid; int ldr;            // optional float32 addend (D may alias it)
   int accumulate;                         // D += (float32 output only)
+  // fused gated-GELU epilogues (CTA-pair kernel, bf16):
+  //   epi 1 (forward): B = [Wi0; Wi1] stored [2F, K]; D = h [M, 2F] receives a = A Wi0^T and b = A Wi1^T, aux = hg [M, F]
+  //                    receives gelu(a) * b.  N must be 2F.
+  //   epi 2 (backward): the product is d(hg) [M, F] (N = F); aux = h [M, 2F] (a | b); D = dh [M, 2F] receives
+  //                    da = d(hg) * b * gelu'(a) and db = d(hg) * gelu(a).
+  int epi; void* aux; int ld_aux; int F;
   int pair;                               // 1: 256 x 256 tiles on CTA pairs (cta_group::2) where M, N >= 256
   int* sk_flags;                          // optional: >= 160 zeroed ints; lets the tcgen05 kernel split the
                                           // tiles of a partial last wave along K over all SMs (float32 output)
@@ -71,6 +77,7 @@ cudaError_t gemm_simt(int dtype, const GemmArgs& g, cudaStream_t st);
 // bounded wait inside the kernel ran out.
 cudaError_t gemm_tc(const GemmArgs& g, int* d_status, cudaStream_t st);
 bool gemm_tc_supported(const GemmArgs& g);
+bool gemm_tc_epi_supported(const GemmArgs& g);   // g.epi != 0 can run fused
 
 struct AttnArgs {
   // rows of Q/O/dQ/dO are (b*Tq + i), rows of K/V/dK/dV are (b*Tk + j);

@@ -38,6 +38,9 @@ struct Params {
   int accumulate;
   int tiles_m, tiles_n;
   int* status;
+  int epi;            // 0 plain, 1 gated-GELU forward, 2 gated-GELU backward (see GemmArgs)
+  void* aux;
+  int ld_aux, F;
   // stream-K tail: the first sk_full * gridDim.x tiles are walked tile by tile; the remaining sk_rem tiles
   // (a partial wave) are cut along K into gridDim.x equal ranges of k-blocks.  sk_rem = 0 turns it off.
   int sk_full, sk_rem;
@@ -159,6 +162,115 @@ __device__ __forceinline__ void store_tile(const Params& p, float* tbuf, uint32_
       }
     }
     __syncwarp();                          // the tile is rewritten by the next chunk
+  }
+}
+
+// ---- gated-GELU epilogues (tanh approximation through the hardware tanh; outputs are bf16)
+__device__ __forceinline__ void gelu_both_fast(float u, float& g, float& dg) {
+  const float c = 0.7978845608028654f, a = 0.044715f;
+  float u2 = u * u, t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(c * (u + a * u * u2)));
+  g = 0.5f * u * (1.f + t);
+  dg = 0.5f * (1.f + t) + 0.5f * u * (1.f - t * t) * c * (1.f + 3.f * a * u2);
+}
+__device__ __forceinline__ void store_bf16x4(bf16* d, float4 v) {
+  __nv_bfloat162 b0 = __floats2bfloat162_rn(v.x, v.y), b1 = __floats2bfloat162_rn(v.z, v.w);
+  uint2 o;
+  o.x = *reinterpret_cast<uint32_t*>(&b0);
+  o.y = *reinterpret_cast<uint32_t*>(&b1);
+  *reinterpret_cast<uint2*>(d) = o;
+}
+__device__ __forceinline__ float4 load_bf16x4(const bf16* p) {
+  uint2 u = *reinterpret_cast<const uint2*>(p);
+  return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                     __uint_as_float(u.y & 0xffff0000u));
+}
+// one accumulator chunk (32 columns of this thread's row) -> the warp's coalesced layout (8 x float4 per lane)
+__device__ __forceinline__ void transpose_chunk(float* tbuf, int lane, const uint32_t (&r)[32], float alpha, float4 (&v)[8]) {
+  const int rr0 = lane >> 3, cc = (lane & 7) * 4;
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    *reinterpret_cast<float4*>(tbuf + lane * 36 + j * 4) =
+        make_float4(alpha * __uint_as_float(r[4 * j]), alpha * __uint_as_float(r[4 * j + 1]),
+                    alpha * __uint_as_float(r[4 * j + 2]), alpha * __uint_as_float(r[4 * j + 3]));
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 8; ++i) v[i] = *reinterpret_cast<const float4*>(tbuf + (i * 4 + rr0) * 36 + cc);
+  __syncwarp();
+}
+// forward: accumulator columns [0,128) = a, [128,256) = b of feature block tn; writes h = [a | b] and hg = gelu(a) b
+__device__ __forceinline__ void store_tile_geglu_fwd(const Params& p, float* tbuf, uint32_t tacc, int m0, int tn, int quad,
+                                                     int lane) {
+  const int rr0 = lane >> 3, cc = (lane & 7) * 4;
+  bf16* H = (bf16*)p.D;
+  bf16* HG = (bf16*)p.aux;
+#pragma unroll 1
+  for (int c = 0; c < 4; ++c) {
+    uint32_t ra[32], rb[32];
+    tmem_ld_32x32b_x32(tacc + c * 32, ra);
+    tmem_ld_32x32b_x32(tacc + 128 + c * 32, rb);
+    tmem_wait_ld_dep(ra);
+    tmem_wait_ld_dep(rb);
+    float4 va[8], vb[8];
+    transpose_chunk(tbuf, lane, ra, p.alpha, va);
+    transpose_chunk(tbuf, lane, rb, p.alpha, vb);
+    const int col = tn * 128 + c * 32 + cc;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int row = m0 + quad * 32 + i * 4 + rr0;
+      if (row < p.M && col < p.F) {
+        store_bf16x4(H + (int64_t)row * p.ldd + col, va[i]);
+        store_bf16x4(H + (int64_t)row * p.ldd + p.F + col, vb[i]);
+        // the product uses a and b as stored (rounded to bf16): the backward pass recomputes from those
+        auto rb = [](float x) { return __bfloat162float(__float2bfloat16_rn(x)); };
+        const float4 a = make_float4(rb(va[i].x), rb(va[i].y), rb(va[i].z), rb(va[i].w));
+        const float4 b = make_float4(rb(vb[i].x), rb(vb[i].y), rb(vb[i].z), rb(vb[i].w));
+        float g0, g1, g2, g3, t;
+        gelu_both_fast(a.x, g0, t); gelu_both_fast(a.y, g1, t); gelu_both_fast(a.z, g2, t); gelu_both_fast(a.w, g3, t);
+        store_bf16x4(HG + (int64_t)row * p.ld_aux + col, make_float4(g0 * b.x, g1 * b.y, g2 * b.z, g3 * b.w));
+      }
+    }
+  }
+}
+// backward: the accumulator is d(hg); aux = h = [a | b]; writes dh = [d(hg) b gelu'(a) | d(hg) gelu(a)]
+template <int BN>
+__device__ __forceinline__ void store_tile_geglu_bwd(const Params& p, float* tbuf, uint32_t tacc, int m0, int n0, int quad,
+                                                     int lane) {
+  const int rr0 = lane >> 3, cc = (lane & 7) * 4;
+  const bf16* Hh = (const bf16*)p.aux;
+  bf16* DH = (bf16*)p.D;
+#pragma unroll 1
+  for (int c = 0; c < BN / 32; ++c) {
+    if (n0 + c * 32 >= p.N) break;
+    uint32_t r[32];
+    tmem_ld_32x32b_x32(tacc + c * 32, r);
+    tmem_wait_ld_dep(r);
+    const int col = n0 + c * 32 + cc;
+    float4 av[8], bv[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {      // a and b of the same elements, in flight while the chunk is transposed
+      const int row = m0 + quad * 32 + i * 4 + rr0;
+      const bool in = row < p.M && col < p.N;
+      av[i] = in ? load_bf16x4(Hh + (int64_t)row * p.ld_aux + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+      bv[i] = in ? load_bf16x4(Hh + (int64_t)row * p.ld_aux + p.F + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float4 v[8];
+    transpose_chunk(tbuf, lane, r, p.alpha, v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int row = m0 + quad * 32 + i * 4 + rr0;
+      if (row < p.M && col < p.N) {
+        // d(hg) is rounded to bf16 first, as when it is stored between two kernels
+        float4 g = make_float4(__bfloat162float(__float2bfloat16_rn(v[i].x)), __bfloat162float(__float2bfloat16_rn(v[i].y)),
+                               __bfloat162float(__float2bfloat16_rn(v[i].z)), __bfloat162float(__float2bfloat16_rn(v[i].w)));
+        float ge[4], dge[4];
+        gelu_both_fast(av[i].x, ge[0], dge[0]); gelu_both_fast(av[i].y, ge[1], dge[1]);
+        gelu_both_fast(av[i].z, ge[2], dge[2]); gelu_both_fast(av[i].w, ge[3], dge[3]);
+        store_bf16x4(DH + (int64_t)row * p.ldd + col,
+                     make_float4(g.x * bv[i].x * dge[0], g.y * bv[i].y * dge[1], g.z * bv[i].z * dge[2], g.w * bv[i].w * dge[3]));
+        store_bf16x4(DH + (int64_t)row * p.ldd + p.F + col, make_float4(g.x * ge[0], g.y * ge[1], g.z * ge[2], g.w * ge[3]));
+      }
+    }
   }
 }
 
@@ -405,7 +517,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       while (ok && wi.next(w)) {
         int tm, tn;
         tile_coords(w.tile, p.tiles_m, p.tiles_n, tm, tn);
-        const int m0 = tm * 256 + (int)rank * 128, n0 = tn * 256 + (int)rank * 128;
+        const int m0 = tm * 256 + (int)rank * 128;
+        // B rows of this CTA: its half of the 256-column tile, or (gated-GELU forward) the Wi0 / Wi1 block
+        const int n0 = p.epi == 1 ? (int)rank * p.F + tn * 128 : tn * 256 + (int)rank * 128;
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status, 6)) { ok = false; break; }
           unsigned char* sa = smem + s * S::kStageBytes;
@@ -492,8 +606,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      store_tile<BN>(p, reinterpret_cast<float*>(smem + S::kEpiOffset) + quad * (32 * 36),
-                     tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16), m0, n0, quad, lane, w.kind == 2);
+      float* tb = reinterpret_cast<float*>(smem + S::kEpiOffset) + quad * (32 * 36);
+      const uint32_t tacc = tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16);
+      if (p.epi == 1) store_tile_geglu_fwd(p, tb, tacc, m0, tn, quad, lane);
+      else if (p.epi == 2) store_tile_geglu_bwd<BN>(p, tb, tacc, m0, n0, quad, lane);
+      else store_tile<BN>(p, tb, tacc, m0, n0, quad, lane, w.kind == 2);
       if (w.kind == 1) {
         __threadfence();
         __syncwarp();
@@ -559,6 +676,7 @@ cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& 
   p.M = g.M; p.N = g.N; p.K = g.K; p.alpha = g.alpha; p.D = g.D; p.ldd = g.ldd; p.out_f32 = g.out_f32;
   p.resid = g.resid; p.ldr = g.ldr; p.accumulate = g.accumulate;
   p.tiles_m = (g.M + BM - 1) / BM; p.tiles_n = (g.N + BN - 1) / BN; p.status = status;
+  p.epi = 0; p.aux = nullptr; p.ld_aux = 0; p.F = 0;
   int tiles = p.tiles_m * p.tiles_n;
   int grid = tiles < g_num_sms ? tiles : g_num_sms;
   p.sk_full = 0; p.sk_rem = 0; p.sk_flags = nullptr;
@@ -587,13 +705,14 @@ cudaError_t launch2(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap&
   Params p;
   p.M = g.M; p.N = g.N; p.K = g.K; p.alpha = g.alpha; p.D = g.D; p.ldd = g.ldd; p.out_f32 = g.out_f32;
   p.resid = g.resid; p.ldr = g.ldr; p.accumulate = g.accumulate;
-  p.tiles_m = (g.M + 255) / 256; p.tiles_n = (g.N + 255) / 256; p.status = status;
+  p.tiles_m = (g.M + 255) / 256; p.tiles_n = g.epi == 1 ? g.F / 128 : (g.N + 255) / 256; p.status = status;
+  p.epi = g.epi; p.aux = g.aux; p.ld_aux = g.ld_aux; p.F = g.F;
   p.sk_full = 0; p.sk_rem = 0; p.sk_flags = nullptr;
   int tiles = p.tiles_m * p.tiles_n;
   int pairs = g_num_sms / 2;
   const int k_blocks = (g.K + BK - 1) / BK, rem = tiles % pairs;
   // long-K float32-output GEMMs: split the tiles of a partial last wave along K over all pairs
-  if (g.sk_flags && g.out_f32 && rem > 0 && k_blocks >= 128 && tiles >= pairs && pairs <= 160 &&
+  if (g.epi == 0 && g.sk_flags && g.out_f32 && rem > 0 && k_blocks >= 128 && tiles >= pairs && pairs <= 160 &&
       (pairs - rem) * 8 > pairs * (tiles / pairs + 1)) {
     p.sk_full = tiles / pairs; p.sk_rem = rem; p.sk_flags = g.sk_flags;
   } else if (tiles < pairs) {
@@ -643,9 +762,19 @@ bool gemm_tc_supported(const GemmArgs& g) {
   return tc::get_encode() != nullptr;
 }
 
+bool gemm_tc_epi_supported(const GemmArgs& g) {
+  if (g.epi != 1 && g.epi != 2) return false;
+  auto al16 = [](const void* p) { return ((uintptr_t)p & 15) == 0; };
+  if (!g.pair || g.out_f32 || g.resid || g.accumulate || g.M < 256 || !g.aux || !al16(g.aux)) return false;
+  if (g.F < 128 || g.F % 128 || g.ld_aux % 8 || g.ldd % 8) return false;
+  if (g.epi == 1) return g.a_kmajor && g.b_kmajor && g.N == 2 * g.F && g.ldd >= 2 * g.F && g.ld_aux >= g.F;
+  return g.N == g.F && g.ldd >= 2 * g.F && g.ld_aux >= 2 * g.F;
+}
+
 cudaError_t gemm_tc(const GemmArgs& g, int* d_status, cudaStream_t st) {
   g_num_sms = num_sms_of_current_device();
   if (g_num_sms <= 0) return cudaErrorInvalidDevice;
+  if (g.epi != 0) return gemm_tc_epi_supported(g) ? dispatch2(g, d_status, st) : cudaErrorInvalidValue;
   if (g.pair && g.M >= 256 && g.N >= 256) return dispatch2(g, d_status, st);
   // wide tiles unless N is small enough that they would mostly compute padding
   if (g.N > 128) return dispatch<256, 4>(g, d_status, st);

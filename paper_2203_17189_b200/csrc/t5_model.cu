@@ -302,7 +302,7 @@ void gemm(Ctx& cx, const GemmArgs& g0, const char* what) {
   g.pair = ((cx.h->cfg.flags >> 2) & 1) ^ 1;      // CTA pairs unless flag bit 2 says otherwise
   if (g.out_f32 && cx.sk_next < kSkSlices) g.sk_flags = cx.w->sk_flags + (cx.sk_next++) * kSkSliceInts;
   ProfScope ps(cx, CAT_GEMM, 2.0 * g.M * g.N * g.K, 1);
-  if (dt == DT_BF16 && !(cx.h->cfg.flags & 1) && gemm_tc_supported(g)) {
+  if (g.epi != 0 || (dt == DT_BF16 && !(cx.h->cfg.flags & 1) && gemm_tc_supported(g))) {
     CK(gemm_tc(g, cx.w->status, cx.st), what);
   } else {
     CK(gemm_simt(dt, g, cx.st), what);
@@ -448,16 +448,33 @@ void attn_backward(Ctx& cx, const AttnP& p, const AttnWs& a, float* dX, void* dX
   dbg_round(cx, dXb, (int64_t)Nq * d, RB_DXB);
 }
 
+// the gated-GELU epilogues run in the tensor-core GEMM on CTA pairs; flags bit 3 keeps the separate kernels
+bool fused_geglu_ok(Ctx& cx, GemmArgs& g) {
+  const t5_config& c = cx.h->cfg;
+  if (c.dtype != DT_BF16 || (c.flags & (1 | 4 | 8))) return false;
+  g.pair = 1;
+  return gemm_tc_supported(g) && gemm_tc_epi_supported(g);
+}
+
 void ffn_forward(Ctx& cx, const FfnP& p, const FfnWs& f, float* x_out, int64_t N) {
   const t5_config& c = cx.h->cfg;
   int d = c.d_model, F = c.d_ff, dt = c.dtype;
   CKL(CAT_NORM, 1, launch_rmsnorm_fwd(dt, f.x, pptr(cx.h, cx.params, p.norm), f.y, f.rstd, (int)N, d, c.rms_eps, cx.st),
      "rmsnorm_fwd");
   dbg_round(cx, f.y, N * d, RB_Y);
-  proj_fwd(cx, f.y, d, p.wi0, (int)N, 2 * F, d, f.h, 2 * F, 1.f, nullptr, "wi proj");
-  dbg_round(cx, f.h, N * 2 * F, RB_H);
-  CKL(CAT_GEGLU, 1, launch_geglu_fwd(dt, f.h, f.hg, (int)N, F, cx.st), "geglu_fwd");
-  dbg_round(cx, f.hg, N * F, RB_HG);
+  GemmArgs gf{};
+  gf.M = (int)N; gf.N = 2 * F; gf.K = d; gf.alpha = 1.f;
+  gf.A = f.y; gf.lda = d; gf.a_kmajor = 1;
+  gf.B = pptr(cx.h, cx.params, p.wi0); gf.ldb = d; gf.b_kmajor = 1;
+  gf.D = f.h; gf.ldd = 2 * F; gf.epi = 1; gf.aux = f.hg; gf.ld_aux = F; gf.F = F;
+  if (fused_geglu_ok(cx, gf)) {
+    gemm(cx, gf, "wi proj + gated GELU");
+  } else {
+    proj_fwd(cx, f.y, d, p.wi0, (int)N, 2 * F, d, f.h, 2 * F, 1.f, nullptr, "wi proj");
+    dbg_round(cx, f.h, N * 2 * F, RB_H);
+    CKL(CAT_GEGLU, 1, launch_geglu_fwd(dt, f.h, f.hg, (int)N, F, cx.st), "geglu_fwd");
+    dbg_round(cx, f.hg, N * F, RB_HG);
+  }
   proj_fwd(cx, f.hg, F, p.wo, (int)N, d, F, x_out, d, 1.f, f.x, "wo proj");
 }
 
@@ -466,10 +483,19 @@ void ffn_backward(Ctx& cx, const FfnP& p, const FfnWs& f, float* dX, void* dXb, 
   Workspace& w = *cx.w;
   int d = c.d_model, F = c.d_ff, dt = c.dtype, n = (int)N;
   proj_wgrad(cx, dXb, d, f.hg, F, p.wo, n, d, F, 1.f, "wgrad ffn.wo");
-  proj_dgrad(cx, dXb, d, p.wo, n, d, F, w.dhg, F, 1.f, 0, 0, "dgrad ffn.wo");
-  dbg_round(cx, w.dhg, N * F, RB_DHG);
-  CKL(CAT_GEGLU, 1, launch_geglu_bwd(dt, w.dhg, f.h, w.dh, n, F, cx.st), "geglu_bwd");
-  dbg_round(cx, w.dh, N * 2 * F, RB_DH);
+  GemmArgs gb{};
+  gb.M = n; gb.N = F; gb.K = d; gb.alpha = 1.f;
+  gb.A = dXb; gb.lda = d; gb.a_kmajor = 1;
+  gb.B = pptr(cx.h, cx.params, p.wo); gb.ldb = F; gb.b_kmajor = 0;
+  gb.D = w.dh; gb.ldd = 2 * F; gb.epi = 2; gb.aux = f.h; gb.ld_aux = 2 * F; gb.F = F;
+  if (fused_geglu_ok(cx, gb)) {
+    gemm(cx, gb, "dgrad ffn.wo + gated GELU backward");
+  } else {
+    proj_dgrad(cx, dXb, d, p.wo, n, d, F, w.dhg, F, 1.f, 0, 0, "dgrad ffn.wo");
+    dbg_round(cx, w.dhg, N * F, RB_DHG);
+    CKL(CAT_GEGLU, 1, launch_geglu_bwd(dt, w.dhg, f.h, w.dh, n, F, cx.st), "geglu_bwd");
+    dbg_round(cx, w.dh, N * 2 * F, RB_DH);
+  }
   proj_wgrad(cx, w.dh, 2 * F, f.y, d, p.wi0, n, 2 * F, d, 1.f, "wgrad ffn.wi");
   proj_dgrad(cx, w.dh, 2 * F, p.wi0, n, 2 * F, d, w.dy, d, 1.f, 0, 0, "dgrad ffn.wi");
   dbg_round(cx, w.dy, N * d, RB_DY);
