@@ -73,6 +73,8 @@ typedef struct {
                                GEMM kernel, bit 1 = use the plain SIMT attention kernels,
                                bit 2 = do NOT run the GEMMs on CTA pairs (cta_group::2),
                                bit 3 = keep the gated GELU in separate kernels instead of the GEMM epilogues.
+                               bit 17 = attention backward as two kernels that each recompute the scores
+                               (no dS scratch in the workspace) instead of the one-pass pair.
                                In float32 mode bits 4..16 round one family of intermediates
                                to bfloat16 in place (normed activations, projections, context,
                                FFN pre-activations, gated product, logits, dlogits, residual
@@ -215,6 +217,28 @@ T5_API int t5_attention(int32_t dtype, int32_t impl, int32_t backward, int32_t B
                         const float* d_bias_delta, const void* d_do, int32_t lddo, void* d_dq, int32_t lddq,
                         void* d_dk, int32_t lddk, void* d_dv, int32_t lddv, float* d_delta,
                         float* d_dbias_delta, void* stream);
+
+/* Attention backward in one pass over the scores (tcgen05 kernels, bfloat16,
+ * d_kv 64): the same result as t5_attention(..., backward = 1, ...) - whose two
+ * kernels each recompute the scores and the probabilities - from one kernel that
+ * produces dK, dV and a bfloat16 copy of dS^T in d_ds_scratch, and a second that
+ * takes dQ = scale dS K from that copy.  (Backward of the attention the
+ * "Example Models" section's T5 family uses.)  d_ds_scratch: device buffer of at
+ * least t5_attention_ds_scratch_bytes(B, H, Tq, Tk) bytes, 128-byte aligned,
+ * owned by the caller, contents undefined on return.  bias_far: 0, or a distance
+ * F such that the bias is constant for (j - i) >= F and for (j - i) <= -F; the
+ * dS mass of those regions is then added to the entries at +F and -F of
+ * d_dbias_delta.  Other arguments as in t5_attention.  T5_ERR_ARG if the shape is
+ * not covered (d_kv != 64, or a query length whose per-CTA tables exceed shared
+ * memory) or the scratch is too small. */
+T5_API int t5_attention_ds_scratch_bytes(int32_t B, int32_t H, int32_t Tq, int32_t Tk, int64_t* bytes);
+T5_API int t5_attention_backward_onepass(
+    int32_t B, int32_t H, int32_t Tq, int32_t Tk, int32_t d_kv, int32_t causal, float scale, const void* d_q,
+    int32_t ldq, const void* d_k, int32_t ldk, const void* d_v, int32_t ldv, const void* d_o, int32_t ldo,
+    const float* d_o32, const float* d_lse, const int32_t* d_code_q, const int32_t* d_code_k,
+    const float* d_bias_delta, const void* d_do, int32_t lddo, void* d_dq, int32_t lddq, void* d_dk, int32_t lddk,
+    void* d_dv, int32_t lddv, float* d_delta, float* d_dbias_delta, int32_t bias_far, void* d_ds_scratch,
+    int64_t ds_scratch_bytes, void* stream);
 
 /* Attention backward without caller-provided scratch.  The paper has no
  * counterpart; this exists for callers that cannot allocate device memory:

@@ -42,7 +42,8 @@ EXPORTS = ["t5_create", "t5_destroy", "t5_last_error", "t5_param_count", "t5_par
            "t5_param_manifest", "t5_workspace_bytes", "t5_init_params", "t5_train_step_fwd_bwd",
            "t5_encode", "t5_decode_logits", "t5_device_status", "t5_profile_enable", "t5_profile_read",
            "t5_launch_count", "t5_relpos_buckets", "t5_xent_zloss",
-           "t5_gemm", "t5_attention", "t5_attention_backward_noalloc"]
+           "t5_gemm", "t5_attention", "t5_attention_backward_noalloc",
+           "t5_attention_ds_scratch_bytes", "t5_attention_backward_onepass"]
 
 _lib = None
 
@@ -86,6 +87,9 @@ def lib():
                                    + [vp, i32] * 4 + [vp, vp, vp])
         L.t5_attention_backward_noalloc.argtypes = ([i32] * 8 + [f32] + [vp, i32] * 4 + [vp] * 5
                                                     + [vp, i32] * 4 + [vp, vp])
+        L.t5_attention_ds_scratch_bytes.argtypes = [i32] * 4 + [C.POINTER(i64)]
+        L.t5_attention_backward_onepass.argtypes = ([i32] * 6 + [f32] + [vp, i32] * 4 + [vp] * 5
+                                                    + [vp, i32] * 4 + [vp, vp, i32, vp, i64, vp])
         for n in EXPORTS:
             if n != "t5_last_error":
                 getattr(L, n).restype = C.c_int
@@ -255,6 +259,25 @@ def t5_attention(impl, backward, B, H, Tq, Tk, d_kv, causal, scale, q, k, v, o, 
                               _ptr(q), ld(q), _ptr(k), ld(k), _ptr(v), ld(v), _ptr(o), ld(o), _ptr(o32), _ptr(lse),
                               _ptr(code_q), _ptr(code_k), _ptr(bias_delta), _ptr(do), ld(do), _ptr(dq), ld(dq),
                               _ptr(dk), ld(dk), _ptr(dv), ld(dv), _ptr(delta), _ptr(dbias_delta), _stream()))
+
+
+def t5_attention_ds_scratch_bytes(B, H, Tq, Tk):
+    n = C.c_int64()
+    _check(lib().t5_attention_ds_scratch_bytes(B, H, Tq, Tk, C.byref(n)))
+    return n.value
+
+
+def t5_attention_backward_onepass(B, H, Tq, Tk, d_kv, causal, scale, q, k, v, o, o32, lse, code_q, code_k,
+                                  bias_delta, do, dq, dk, dv, delta, dbias_delta, bias_far, ds_scratch):
+    """Attention backward that visits the scores once (dK, dV and a stored dS, then dQ from it)."""
+    _check(lib().t5_attention_backward_onepass(B, H, Tq, Tk, d_kv, int(causal), scale,
+                                               _ptr(q), q.stride(0), _ptr(k), k.stride(0), _ptr(v), v.stride(0),
+                                               _ptr(o), o.stride(0), _ptr(o32), _ptr(lse), _ptr(code_q),
+                                               _ptr(code_k), _ptr(bias_delta), _ptr(do), do.stride(0),
+                                               _ptr(dq), dq.stride(0), _ptr(dk), dk.stride(0), _ptr(dv),
+                                               dv.stride(0), _ptr(delta), _ptr(dbias_delta), int(bias_far),
+                                               _ptr(ds_scratch), ds_scratch.numel() * ds_scratch.element_size(),
+                                               _stream()))
 
 
 def t5_attention_backward_noalloc(impl, B, H, Tq, Tk, d_kv, causal, scale, q, k, v, o, o32, lse, code_q, code_k,

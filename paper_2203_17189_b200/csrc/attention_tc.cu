@@ -50,8 +50,6 @@ struct TcParams {
   int bias_far;              // see AttnArgs::bias_far
 };
 
-__device__ __forceinline__ uint64_t desc_k(uint32_t addr) { return make_desc(addr, 16, 1024); }
-__device__ __forceinline__ uint64_t desc_mn(uint32_t addr, uint32_t lbo) { return make_desc(addr, lbo, 1024); }
 
 // Writes 8 consecutive bf16 of row `row` (columns [col8*8, col8*8+8) of a 64-column chunk) into a
 // 128-byte-swizzled K-major tile: 16-byte piece index is XORed with (row % 8).
@@ -83,17 +81,17 @@ __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u 
 
 // dst[i] = f(i) for i in [0, n) by NT threads; four loads are in flight before their stores, so the
 // set-up of a CTA costs a couple of global-memory round trips instead of one per element.
-template <int NT, typename T, typename F>
+template <int NT, typename T, typename F, int U = 4>
 __device__ __forceinline__ void fill_batched(T* dst, int n, int tid, F f) {
-  for (int base = tid; base < n; base += 4 * NT) {
-    T v[4];
+  for (int base = tid; base < n; base += U * NT) {
+    T v[U];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < U; ++u) {
       int i = base + u * NT;
       if (i < n) v[u] = f(i);
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < U; ++u) {
       int i = base + u * NT;
       if (i < n) dst[i] = v[u];
     }
@@ -161,8 +159,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem;
-  const uint32_t sQ = smem_u32(smem + L::kQ), sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV),
-                 sP = smem_u32(smem + L::kPo);
+  // low words of the operand descriptors (K-major Q, K, P; MN-major V)
+  const uint32_t lQ = desc_lo_k(smem_u32(smem + L::kQ)), lK = desc_lo_k(smem_u32(smem + L::kK)),
+                 lV = desc_lo_mn(smem_u32(smem + L::kV)), lP = desc_lo_k(smem_u32(smem + L::kPo));
   uint64_t* bar_k = &bars->ld[0];
   uint64_t* bar_v = &bars->ld[1];
   uint64_t* bar_m = &bars->mma[0];
@@ -190,8 +189,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
     tc_fence_after();
 #pragma unroll
     for (int kk = 0; kk < DK / 16; ++kk)
-      umma_bf16(tmem_base, desc_k(sQ + (kk >> 2) * 16384 + (kk & 3) * 32), desc_k(sK + (kk >> 2) * 8192 + (kk & 3) * 32),
-                idesc_s, kk != 0);
+      umma_bf16_lo(tmem_base, lQ + (((kk >> 2) * 16384 + (kk & 3) * 32) >> 4), lK + (((kk >> 2) * 8192 + (kk & 3) * 32) >> 4),
+                   idesc_s, kk != 0);
     return true;
   };
 
@@ -306,7 +305,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
-          umma_bf16(tmem_base + 64, desc_k(sP + ks * 32), desc_mn(sV + ks * 2048, 8192), idesc_pv, (t | ks) != 0);
+          umma_bf16_lo(tmem_base + 64, lP + ((ks * 32) >> 4), lV + ((ks * 2048) >> 4), idesc_pv, (t | ks) != 0);
         if (t + 1 < n_kt) good = issue_s();
         if (good) umma_commit(bar_m);
       }
@@ -438,7 +437,8 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem;
-  const uint32_t sQ = smem_u32(smem + L::kQ), sDO = smem_u32(smem + L::kDO), sDS = smem_u32(smem + L::kDS);
+  const uint32_t lQ = desc_lo_k(smem_u32(smem + L::kQ)), lDO = desc_lo_k(smem_u32(smem + L::kDO)),
+                 lDS = desc_lo_k(smem_u32(smem + L::kDS));      // low words of the operand descriptors
 
   const int i = q0 + row;
   const bool row_in = i < p.Tq;
@@ -459,16 +459,16 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
     if (!mbar_wait(&bar_kv[st], ph_kv[st], abort_flag, p.status, 22)) return false;
     ph_kv[st] ^= 1;
     tc_fence_after();
-    const uint32_t sK = smem_u32(smem + L::kKV0 + st * L::kStage), sV = sK + L::kKVTile;
+    const uint32_t lK = desc_lo_k(smem_u32(smem + L::kKV0 + st * L::kStage)), lV = lK + (L::kKVTile >> 4);
 #pragma unroll
     for (int kk = 0; kk < DK / 16; ++kk) {
       uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
-      umma_bf16(tmem_base, desc_k(sQ + oa), desc_k(sK + ob), idesc_s, kk != 0);
+      umma_bf16_lo(tmem_base, lQ + (oa >> 4), lK + (ob >> 4), idesc_s, kk != 0);
     }
 #pragma unroll
     for (int kk = 0; kk < DK / 16; ++kk) {
       uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
-      umma_bf16(tmem_base + 64, desc_k(sDO + oa), desc_k(sV + ob), idesc_s, kk != 0);
+      umma_bf16_lo(tmem_base + 64, lDO + (oa >> 4), lV + (ob >> 4), idesc_s, kk != 0);
     }
     return true;
   };
@@ -564,10 +564,10 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
     __syncthreads();
     if (tid == 0) {
       tc_fence_after();
-      const uint32_t sK = smem_u32(smem + L::kKV0 + (t % 3) * L::kStage);
+      const uint32_t lKm = desc_lo_mn(smem_u32(smem + L::kKV0 + (t % 3) * L::kStage));
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks)
-        umma_bf16(tmem_base + 128, desc_k(sDS + ks * 32), desc_mn(sK + ks * 2048, 8192), idesc_dq, (t | ks) != 0);
+        umma_bf16_lo(tmem_base + 128, lDS + ((ks * 32) >> 4), lKm + ((ks * 2048) >> 4), idesc_dq, (t | ks) != 0);
       bool good = true;
       if (t + 1 < n_kt) good = issue_s_dp(t + 1);      // the scores of tile t are in registers by now
       if (good) umma_commit(bar_m);
@@ -715,8 +715,8 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem;
-  const uint32_t sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV), sPt = smem_u32(smem + L::kPt),
-                 sDSt = smem_u32(smem + L::kDSt);
+  const uint32_t lK = desc_lo_k(smem_u32(smem + L::kK)), lV = desc_lo_k(smem_u32(smem + L::kV)),
+                 lPt = desc_lo_k(smem_u32(smem + L::kPt)), lDSt = desc_lo_k(smem_u32(smem + L::kDSt));
   const int j = k0 + row;
   const bool row_in = j < p.Tk;
   const int ck = row_in ? p.code_k[b * p.Tk + j] : 0;
@@ -732,16 +732,16 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
     if (!mbar_wait(&bar_qd[st], ph_qd[st], abort_flag, p.status, 32)) return false;
     ph_qd[st] ^= 1;
     tc_fence_after();
-    const uint32_t sQ = smem_u32(smem + L::kQD0 + st * L::kStage), sDO = sQ + L::kQTile;
+    const uint32_t lQ = desc_lo_k(smem_u32(smem + L::kQD0 + st * L::kStage)), lDO = lQ + (L::kQTile >> 4);
 #pragma unroll
     for (int kk = 0; kk < DK / 16; ++kk) {
       uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
-      umma_bf16(tmem_base, desc_k(sK + oa), desc_k(sQ + ob), idesc_s, kk != 0);
+      umma_bf16_lo(tmem_base, lK + (oa >> 4), lQ + (ob >> 4), idesc_s, kk != 0);
     }
 #pragma unroll
     for (int kk = 0; kk < DK / 16; ++kk) {
       uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
-      umma_bf16(tmem_base + 64, desc_k(sV + oa), desc_k(sDO + ob), idesc_s, kk != 0);
+      umma_bf16_lo(tmem_base + 64, lV + (oa >> 4), lDO + (ob >> 4), idesc_s, kk != 0);
     }
     return true;
   };
@@ -752,7 +752,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
 
   for (int t = t_begin; t < n_qt && ok; ++t) {
     const int qb = t * 64;
-    const uint32_t sQ = smem_u32(smem + L::kQD0 + (t & 1) * L::kStage), sDO = sQ + L::kQTile;
+    const uint32_t lQm = desc_lo_mn(smem_u32(smem + L::kQD0 + (t & 1) * L::kStage)), lDOm = lQm + (L::kQTile >> 4);
     ok = mbar_wait(bar_m, ph_m, abort_flag, p.status, 33);
     ph_m ^= 1;
     if (!ok) break;
@@ -824,11 +824,10 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
       const uint32_t first = (t == t_begin) ? 0u : 1u;
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks)
-        umma_bf16(tmem_base + 128, desc_k(sPt + ks * 32), desc_mn(sDO + ks * 2048, 8192), idesc_acc, first | ks);
+        umma_bf16_lo(tmem_base + 128, lPt + ((ks * 32) >> 4), lDOm + ((ks * 2048) >> 4), idesc_acc, first | ks);
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks)
-        umma_bf16(tmem_base + 128 + DK, desc_k(sDSt + ks * 32), desc_mn(sQ + ks * 2048, 8192), idesc_acc,
-                  first | ks);
+        umma_bf16_lo(tmem_base + 128 + DK, lDSt + ((ks * 32) >> 4), lQm + ((ks * 2048) >> 4), idesc_acc, first | ks);
       bool good = true;
       if (t + 1 < n_qt) good = issue_st(t + 1);        // the scores of tile t are in registers by now
       if (good) umma_commit(bar_m);
@@ -884,30 +883,574 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
 }
 
 // ----------------------------------------------------------------------------- delta = rowsum(dO * O)
+// Thread = 8 consecutive columns of one token row (16 bytes of dO, 32 bytes of the float32 O copy); the DK / 8
+// threads of a head reduce with shuffles.
 template <int DK>
-__global__ void attn_delta_tc_kernel(const bf16* __restrict__ O, int ldo, const float* __restrict__ O32, int ldo32,
-                                     const bf16* __restrict__ dO, int lddo, float* __restrict__ delta, int B, int H,
-                                     int Tq) {
-  int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (gw >= B * Tq * H) return;
-  int h = gw % H, row = gw / H;
-  int b = row / Tq, i = row % Tq;
+__global__ void __launch_bounds__(256)
+attn_delta_tc_kernel(const bf16* __restrict__ O, int ldo, const float* __restrict__ O32, int ldo32,
+                     const bf16* __restrict__ dO, int lddo, float* __restrict__ delta, int B, int H, int Tq) {
+  const int per_row = H * DK / 8;
+  const int64_t gt = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t n_rows = (int64_t)B * Tq;
+  const bool in = gt < n_rows * per_row;        // per_row is a multiple of DK / 8, so a head never straddles the end
+  const int64_t row = in ? gt / per_row : 0;
+  const int col = in ? (int)(gt - row * per_row) * 8 : 0;
   float s = 0.f;
-#pragma unroll
-  for (int c = 0; c < DK / 64; ++c) {
-    int col = h * DK + c * 64 + lane * 2;
-    __nv_bfloat162 g = *reinterpret_cast<const __nv_bfloat162*>(dO + (int64_t)row * lddo + col);
-    float2 fg = __bfloat1622float2(g), fa;
+  if (in) {
+    const uint4 g = *reinterpret_cast<const uint4*>(dO + row * lddo + col);
+    const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
+    float a[8];
     if (O32) {
-      fa = *reinterpret_cast<const float2*>(O32 + (int64_t)row * ldo32 + col);
+      const float4 a0 = *reinterpret_cast<const float4*>(O32 + row * ldo32 + col);
+      const float4 a1 = *reinterpret_cast<const float4*>(O32 + row * ldo32 + col + 4);
+      a[0] = a0.x; a[1] = a0.y; a[2] = a0.z; a[3] = a0.w; a[4] = a1.x; a[5] = a1.y; a[6] = a1.z; a[7] = a1.w;
     } else {
-      fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(O + (int64_t)row * ldo + col));
+      const uint4 o = *reinterpret_cast<const uint4*>(O + row * ldo + col);
+      const uint32_t ow[4] = {o.x, o.y, o.z, o.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { a[2 * i] = bf16_lo(ow[i]); a[2 * i + 1] = bf16_hi(ow[i]); }
     }
-    s += fa.x * fg.x + fa.y * fg.y;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) s += a[2 * i] * bf16_lo(gw[i]) + a[2 * i + 1] * bf16_hi(gw[i]);
   }
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-  if (lane == 0) delta[(int64_t)(b * H + h) * Tq + i] = s;
+  for (int o = DK / 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if (in && (threadIdx.x & (DK / 8 - 1)) == 0) {
+    const int h = col / DK;
+    const int b = (int)(row / Tq), i = (int)(row - (int64_t)b * Tq);
+    delta[(int64_t)(b * H + h) * Tq + i] = s;
+  }
+}
+
+// ============================================================================ backward in one pass over the scores
+// Kernel A (dK, dV and dS): CTA = 128 keys x all queries (64-query tiles), warp-specialised, two CTAs per SM.
+//   warps 0-7 : softmax.  Warp (quad, half) has 32 keys (its tensor-memory lanes) x 32 of the tile's 64 queries,
+//               walked as two passes of 16: P^T and dS^T from the transposed scores S^T = K Q^T and dP^T = V dO^T
+//               in tensor memory, written as bf16 tiles to shared memory; the bias gradient is reduced along
+//               diagonals as in the dQ kernel above.  As soon as a tile's scores are in registers the warps release
+//               the tensor-memory buffer, so the next tile's S^T / dP^T run during this tile's arithmetic.
+//   warp 8    : issues every MMA (all lanes walk the loop, one elected lane executes): S^T / dP^T of tile t+1, then
+//               the accumulating dV += P^T dO and dK += dS^T Q of tile t.
+//   warp 9    : one thread loads the Q / dO tiles (TMA ring) and stores each dS^T tile to global memory (TMA store
+//               out of the same shared-memory tile the dK MMA reads).
+// The second CTA of the SM is at another point of its life: its set-up, its waits and its epilogue overlap this
+// one's arithmetic.
+// Kernel B (dQ): dQ = scale dS K, a plain TMA -> MMA pipeline over the stored dS^T (an MN-major A operand).
+// The scores, the exponentials and dS are computed once instead of once per kernel; the price is one write and
+// one read of dS (bf16) through global memory.
+template <int DK>
+struct KvfLayout {
+  static constexpr int kStages = 2;                             // Q / dO ring
+  static constexpr int kKVBytes = 128 * DK * 2;
+  static constexpr int kK = 0, kV = kKVBytes, kQD0 = 2 * kKVBytes;
+  static constexpr int kQTile = 64 * DK * 2;                    // one Q or dO tile (64 queries)
+  static constexpr int kStage = 2 * kQTile;                     // Q then dO
+  static constexpr int kP0 = kQD0 + kStages * kStage;           // [128 keys x 64 queries] bf16
+  static constexpr int kDS0 = kP0 + 16384;                      // [128 keys x 64 queries] bf16
+  static constexpr int kMisc = kDS0 + 16384;
+  static constexpr int kBarBytes = 128;
+  static int bytes(int Tq, bool want_db) {
+    int tqp = (Tq + 63) / 64 * 64;
+    return kMisc + (tqp + 128) * 4 + 3 * tqp * 4 + (want_db ? (tqp + 128) * 4 : 0) + kBarBytes + 1024 + 64;
+  }
+};
+
+struct KvfBars {
+  uint64_t kv;
+  uint64_t qd_full[2], qd_free[2];
+  uint64_t s_full, s_free, p_full, p_free;
+  uint64_t acc;
+  uint32_t tmem;
+  int abort_flag;
+};
+static_assert(sizeof(KvfBars) <= 128, "barrier block");
+
+constexpr int kKvfThreads = 10 * 32;
+constexpr int kKvfSoftmaxThreads = 8 * 32;
+
+template <int DK>
+__global__ void __launch_bounds__(kKvfThreads, 2)
+attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mdo,
+                       const __grid_constant__ CUtensorMap mk, const __grid_constant__ CUtensorMap mv,
+                       const __grid_constant__ CUtensorMap mds, const __grid_constant__ CUtensorMap mdk_out,
+                       const __grid_constant__ CUtensorMap mdv_out, TcParams p) {
+  static_assert(DK == 64, "the output tiles are staged as one 128-byte-wide tile per tensor");
+  using L = KvfLayout<DK>;
+  constexpr int NST = L::kStages;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const int tqp = (p.Tq + 63) / 64 * 64;
+  const bool want_db = p.dbias_delta != nullptr;
+  float* bias_s = (float*)(smem + L::kMisc);          // [tqp + 128], entry (key row - query + tqp), log2 units
+  float* lse_s = bias_s + tqp + 128;                  // [tqp]  (log2 units)
+  float* dl_s = lse_s + tqp;                          // [tqp]
+  int* codes_s = (int*)(dl_s + tqp);                  // [tqp] query codes
+  float* dbias_s = (float*)(codes_s + tqp);           // [tqp + 128], entry (key row - query + tqp)
+  KvfBars* bars = (KvfBars*)(((uintptr_t)(dbias_s + (want_db ? tqp + 128 : 0)) + 15) & ~(uintptr_t)15);
+  volatile int* abort_flag = &bars->abort_flag;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int b = blockIdx.z, h = blockIdx.y, k0 = blockIdx.x * 128;
+  const int n_qt = (p.Tq + 63) / 64;
+  const int t_begin = p.causal ? k0 / 64 : 0;          // queries before k0 see none of these keys
+  const int n = n_qt - t_begin;                        // tiles this CTA walks
+  constexpr uint32_t kTmemCols = 256;
+  constexpr uint32_t kColS = 0, kColDP = 64, kColDV = 128, kColDK = 128 + DK;
+
+  auto load_qd = [&](int i) {
+    const int st = i % NST, t = t_begin + i;
+    unsigned char* base = smem + L::kQD0 + st * L::kStage;
+    mbar_arrive_expect_tx(&bars->qd_full[st], L::kStage);
+#pragma unroll
+    for (int c = 0; c < DK / 64; ++c) {
+      tma_load_3d(base + c * 8192, &mq, h * DK + c * 64, t * 64, b, &bars->qd_full[st]);
+      tma_load_3d(base + L::kQTile + c * 8192, &mdo, h * DK + c * 64, t * 64, b, &bars->qd_full[st]);
+    }
+  };
+  if (tid == 9 * 32) {      // the loading thread: its first loads go out before the rest of the set-up
+    mbar_init(&bars->kv, 1);
+    for (int i = 0; i < NST; ++i) { mbar_init(&bars->qd_full[i], 1); mbar_init(&bars->qd_free[i], 1); }
+    mbar_init(&bars->s_full, 1);
+    mbar_init(&bars->s_free, 8);         // the softmax warps have the tile's scores in registers
+    mbar_init(&bars->p_full, 8);         // one arrival per softmax warp
+    mbar_init(&bars->p_free, 2);         // the accumulating MMAs are done + the dS store has read the tile
+    mbar_init(&bars->acc, 1);
+    bars->abort_flag = 0;
+    fence_barrier_init();
+    if (n > 0) {
+      mbar_arrive_expect_tx(&bars->kv, 2 * L::kKVBytes);
+#pragma unroll
+      for (int c = 0; c < DK / 64; ++c) {
+        tma_load_3d(smem + L::kK + c * 16384, &mk, h * DK + c * 64, k0, b, &bars->kv);
+        tma_load_3d(smem + L::kV + c * 16384, &mv, h * DK + c * 64, k0, b, &bars->kv);
+      }
+      for (int i = 0; i < NST && i < n; ++i) load_qd(i);
+    }
+  }
+  if (warp == 8) tmem_alloc(&bars->tmem, kTmemCols);
+  const int span = p.Tq + p.Tk - 1;
+  if (warp < 8) {
+    // One batched fill of the four per-CTA tables (contiguous in shared memory), every global load in flight at
+    // once.  Bias: distance of (key j = k0 + row, query q) is j - q, window index w = row - q + tqp in [1, tqp + 127].
+    const int64_t bh = (int64_t)(b * p.H + h) * p.Tq;
+    const int nb = tqp + 128;
+    auto table = [&](int x) -> uint32_t {
+      if (x < nb) {
+        int g = (x - tqp) + k0 + p.Tq - 1;
+        return __float_as_uint((p.bias_delta && g >= 0 && g < span) ? p.bias_delta[(int64_t)h * span + g] * kLog2e : 0.f);
+      }
+      x -= nb;
+      if (x < tqp) return __float_as_uint(x < p.Tq ? p.lse[bh + x] * kLog2e : -INFINITY);
+      x -= tqp;
+      if (x < tqp) return __float_as_uint(x < p.Tq ? p.delta[bh + x] : 0.f);
+      x -= tqp;
+      return (uint32_t)(x < p.Tq ? p.code_q[b * p.Tq + x] : 0);
+    };
+    fill_batched<kKvfSoftmaxThreads, uint32_t, decltype(table), 9>((uint32_t*)bias_s, nb + 3 * tqp, tid, table);
+    if (want_db)
+      for (int w = tid; w < nb; w += kKvfSoftmaxThreads) dbias_s[w] = 0.f;
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem;
+  bool ok = true;
+
+  if (warp == 9) {
+    // ------------------------------------------------------------------ loads and the dS store
+    if (lane == 0 && n > 0) {
+      for (int i = 0; i < n && ok; ++i) {
+        ok = mbar_wait_relaxed(&bars->p_full, i & 1, abort_flag, p.status, 41);
+        if (!ok) break;
+        tma_store_3d(&mds, smem + L::kDS0, (t_begin + i) * 64, k0, b * p.H + h);
+        bulk_commit_group();
+        if (i + NST < n) {    // the reload goes out before the store's read is waited for: its latency is the longer one
+          ok = mbar_wait_relaxed(&bars->qd_free[i % NST], (i / NST) & 1, abort_flag, p.status, 42);
+          if (ok) load_qd(i + NST);
+        }
+        bulk_wait_group_read<0>();                      // the store has read the tile: the softmax warps may refill it
+        mbar_arrive(&bars->p_free);
+      }
+      bulk_wait_group<0>();
+      if (!ok) {   // a wait ran out: give loads still in flight a bounded time to land
+        long long t0 = clock64();
+        while (clock64() - t0 < 4000000ll) {}
+      }
+    }
+  } else if (warp == 8) {
+    // ------------------------------------------------------------------ MMA issue
+    // All 32 lanes walk the loop (waits included) so that its counters and the descriptor words are warp-uniform;
+    // the elected lane alone executes the MMAs and commits.
+    if (n > 0) {
+      const uint32_t lead = elect_one_lane();
+      constexpr uint32_t idesc_s = make_idesc(128, 64, false, false);
+      constexpr uint32_t idesc_acc = make_idesc(128, DK, false, true);
+      // low words of the operand descriptors: K and V (K-major), the Q / dO ring, the P^T / dS^T tiles
+      const uint32_t lK = desc_lo_k(smem_u32(smem + L::kK)), lV = desc_lo_k(smem_u32(smem + L::kV));
+      const uint32_t lQ0 = desc_lo_k(smem_u32(smem + L::kQD0)), lPt = desc_lo_k(smem_u32(smem + L::kP0)),
+                     lDSt = desc_lo_k(smem_u32(smem + L::kDS0));
+      constexpr uint32_t kToMn = ((8192u >> 4) << 16) - ((16u >> 4) << 16);   // K-major low word -> MN-major
+      // S^T = K Q^T and dP^T = V dO^T of tile i
+      auto issue_sdp = [&](int i) {
+        const int st = i % NST;
+        if (!__all_sync(0xffffffffu, mbar_wait_relaxed(&bars->qd_full[st], (i / NST) & 1, abort_flag, p.status, 43))) return false;
+        tc_fence_after();
+        const uint32_t lQ = lQ0 + st * (L::kStage >> 4), lDO = lQ + (L::kQTile >> 4);
+#pragma unroll
+        for (int kk = 0; kk < DK / 16; ++kk) {
+          uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
+          umma_bf16_lo_lead(tmem_base + kColS, lK + (oa >> 4), lQ + (ob >> 4), idesc_s, kk != 0, lead);
+        }
+#pragma unroll
+        for (int kk = 0; kk < DK / 16; ++kk) {
+          uint32_t oa = (kk >> 2) * 16384 + (kk & 3) * 32, ob = (kk >> 2) * 8192 + (kk & 3) * 32;
+          umma_bf16_lo_lead(tmem_base + kColDP, lV + (oa >> 4), lDO + (ob >> 4), idesc_s, kk != 0, lead);
+        }
+        umma_commit_lead(&bars->s_full, lead);
+        return true;
+      };
+      ok = __all_sync(0xffffffffu, mbar_wait_relaxed(&bars->kv, 0, abort_flag, p.status, 44));
+      if (ok) ok = issue_sdp(0);
+      for (int i = 0; i < n && ok; ++i) {
+        const int st = i % NST;
+        if (i + 1 < n) {      // the softmax warps have the scores of tile i in registers: S^T / dP^T of tile i+1 go first
+          ok = __all_sync(0xffffffffu, mbar_wait_relaxed(&bars->s_free, i & 1, abort_flag, p.status, 49));
+          if (!ok) break;
+          tc_fence_after();
+          ok = issue_sdp(i + 1);
+          if (!ok) break;
+        }
+        ok = __all_sync(0xffffffffu, mbar_wait_relaxed(&bars->p_full, i & 1, abort_flag, p.status, 45));
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t lQm = lQ0 + st * (L::kStage >> 4) + kToMn, lDOm = lQm + (L::kQTile >> 4);
+        const uint32_t first = i == 0 ? 0u : 1u;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          umma_bf16_lo_lead(tmem_base + kColDV, lPt + ((ks * 32) >> 4), lDOm + ((ks * 2048) >> 4), idesc_acc, first | ks, lead);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          umma_bf16_lo_lead(tmem_base + kColDK, lDSt + ((ks * 32) >> 4), lQm + ((ks * 2048) >> 4), idesc_acc, first | ks, lead);
+        umma_commit_lead(&bars->p_free, lead);
+        umma_commit_lead(&bars->qd_free[st], lead);
+      }
+      if (ok) umma_commit_lead(&bars->acc, lead);
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax warps
+    const int quad = warp & 3, half = warp >> 2, row = quad * 32 + lane;
+    const int j = k0 + row;
+    const int ck = j < p.Tk ? p.code_k[b * p.Tk + j] : 0;
+    const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
+    const float sc2 = p.scale * kLog2e;
+    const bool has_bias = p.bias_delta != nullptr;
+    float far_pos = 0.f, far_neg = 0.f;
+    unsigned char* tP = smem + L::kP0;
+    unsigned char* tD = smem + L::kDS0;
+    for (int i = 0; i < n && ok; ++i) {
+      const int qb = (t_begin + i) * 64;
+      const uint32_t par = i & 1;
+      ok = mbar_wait_relaxed(&bars->s_full, par, abort_flag, p.status, 46);
+      if (!ok) break;
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        const int cc = half * 32 + c * 16;                 // first of this pass's 16 queries within the tile
+        const int qq0 = qb + cc;
+        int cmine = codes_s[qq0 + (lane & 15)];
+        const bool fast = __all_sync(0xffffffffu, cmine == ck) && ck != 0 &&
+                          (!p.causal || k0 + quad * 32 + 31 <= qq0);           // warp-uniform: no mask needed
+        const float* brow = bias_s + (row - qq0 + tqp);    // element e: brow[-e]
+        uint32_t rs[16], rp[16];
+        tmem_ld_32x32b_x16(tmem_base + lane_off + kColS + cc, rs);
+        tmem_ld_32x32b_x16(tmem_base + lane_off + kColDP + cc, rp);
+        tmem_wait_ld_dep16(rs);
+        tmem_wait_ld_dep16(rp);
+        if (c == 1) {      // both passes are out of tensor memory: the MMA warp may overwrite the buffer (tile i+1)
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars->s_free);
+        }
+        float pt[16], ds[16];
+        auto compute = [&](auto fast_c, auto bias_c) {
+          constexpr bool FAST = decltype(fast_c)::value, BIAS = decltype(bias_c)::value;
+#pragma unroll
+          for (int i4 = 0; i4 < 4; ++i4) {
+            const float4 l4 = *reinterpret_cast<const float4*>(lse_s + qq0 + i4 * 4);
+            const float4 d4 = *reinterpret_cast<const float4*>(dl_s + qq0 + i4 * 4);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int ii = i4 * 4 + e;
+              const float lse2 = e == 0 ? l4.x : e == 1 ? l4.y : e == 2 ? l4.z : l4.w;
+              const float dlq = e == 0 ? d4.x : e == 1 ? d4.y : e == 2 ? d4.z : d4.w;
+              float sv = BIAS ? fmaf(__uint_as_float(rs[ii]), sc2, brow[-ii]) : __uint_as_float(rs[ii]) * sc2;
+              float pr = ex2_approx(sv - lse2);
+              if (!FAST) {
+                int q = qq0 + ii;
+                int cqv = codes_s[q];
+                bool valid = ck != 0 && ck == cqv && (!p.causal || j <= q) && lse2 != -INFINITY;
+                pr = valid ? pr : 0.f;
+              }
+              pt[ii] = pr;
+              ds[ii] = pr * (__uint_as_float(rp[ii]) - dlq);
+            }
+          }
+        };
+        if (fast) {
+          if (has_bias) compute(std::true_type{}, std::true_type{}); else compute(std::true_type{}, std::false_type{});
+        } else {
+          if (has_bias) compute(std::false_type{}, std::true_type{}); else compute(std::false_type{}, std::false_type{});
+        }
+        if (want_db) {
+          const int kk0 = k0 + quad * 32;                  // this pass: 32 keys x 16 queries
+          if (p.bias_far > 0 && kk0 - (qq0 + 15) >= p.bias_far) {
+            float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+            for (int e = 0; e < 16; e += 2) { t0 += ds[e]; t1 += ds[e + 1]; }
+            far_pos += t0 + t1;
+          } else if (p.bias_far > 0 && qq0 - (kk0 + 31) >= p.bias_far) {
+            float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+            for (int e = 0; e < 16; e += 2) { t0 += ds[e]; t1 += ds[e + 1]; }
+            far_neg += t0 + t1;
+          } else {
+            // Diagonal sums of the 32 x 16 block: at step e lane l takes query e of key row (l + e) mod 32, which
+            // lies on diagonal (key - query) = l when l + e < 32 and l - 32 otherwise.
+            float tot = 0.f, a1 = 0.f;
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              float v = __shfl_sync(0xffffffffu, ds[e], lane + e);      // source lane taken modulo 32
+              tot += v;
+              a1 += (lane + e >= 32) ? v : 0.f;
+            }
+            // window entry (key row - query + tqp); warps and passes overlap there: atomics
+            float* win = dbias_s + (quad * 32 + lane - qq0 + tqp);
+            atomicAdd(win, tot - a1);
+            if (lane >= 17) atomicAdd(win - 32, a1);
+          }
+        }
+        if (c == 0) {
+          // the tile buffers are free once the accumulating MMAs of tile i-1 are done and its dS store has read them
+          ok = mbar_wait_relaxed(&bars->p_free, par ^ 1, abort_flag, p.status, 47);
+        }
+        if (ok) {
+#pragma unroll
+          for (int q8 = 0; q8 < 2; ++q8) {
+            uint4 v;
+            v.x = pack_bf16(pt[q8 * 8 + 0], pt[q8 * 8 + 1]);
+            v.y = pack_bf16(pt[q8 * 8 + 2], pt[q8 * 8 + 3]);
+            v.z = pack_bf16(pt[q8 * 8 + 4], pt[q8 * 8 + 5]);
+            v.w = pack_bf16(pt[q8 * 8 + 6], pt[q8 * 8 + 7]);
+            store_swizzled_16B(tP, row, (cc >> 3) + q8, v);
+            v.x = pack_bf16(ds[q8 * 8 + 0], ds[q8 * 8 + 1]);
+            v.y = pack_bf16(ds[q8 * 8 + 2], ds[q8 * 8 + 3]);
+            v.z = pack_bf16(ds[q8 * 8 + 4], ds[q8 * 8 + 5]);
+            v.w = pack_bf16(ds[q8 * 8 + 6], ds[q8 * 8 + 7]);
+            store_swizzled_16B(tD, row, (cc >> 3) + q8, v);
+          }
+        }
+      }
+      if (!ok) break;
+      fence_proxy_async();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->p_full);
+    }
+    if (ok && n > 0) ok = mbar_wait_relaxed(&bars->acc, 0, abort_flag, p.status, 48);
+    // the last dS store must have read its tile before the tile buffers are reused for the output rows
+    if (ok && n > 0) ok = mbar_wait_relaxed(&bars->p_free, (n - 1) & 1, abort_flag, p.status, 50);
+    // every softmax thread gets here whatever happened; behind this barrier the abort flag gives the whole group
+    // one answer, so the barrier inside the epilogue is reached by all of them or by none
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    ok = *abort_flag == 0;
+    if (ok) {
+      tc_fence_after();
+      // dV and dK rows go through the (now idle) P^T / dS^T tiles as 128-byte-swizzled [128 keys x 64] bf16 tiles
+      // and leave with one TMA store each: full 128-byte row segments, rows beyond Tk clipped by the tensor map
+      unsigned char* tV = smem + L::kP0;
+      unsigned char* tK = smem + L::kDS0;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        const int cc = half * 32 + c * 16;
+        uint32_t rv[16], rk[16];
+        if (n > 0) {
+          tmem_ld_32x32b_x16(tmem_base + lane_off + kColDV + cc, rv);
+          tmem_ld_32x32b_x16(tmem_base + lane_off + kColDK + cc, rk);
+          tmem_wait_ld_dep16(rv);
+          tmem_wait_ld_dep16(rk);
+        } else {
+#pragma unroll
+          for (int d = 0; d < 16; ++d) rv[d] = rk[d] = 0u;
+        }
+#pragma unroll
+        for (int q8 = 0; q8 < 2; ++q8) {
+          const int d = q8 * 8;
+          uint4 v;
+          v.x = pack_bf16(__uint_as_float(rv[d]), __uint_as_float(rv[d + 1]));
+          v.y = pack_bf16(__uint_as_float(rv[d + 2]), __uint_as_float(rv[d + 3]));
+          v.z = pack_bf16(__uint_as_float(rv[d + 4]), __uint_as_float(rv[d + 5]));
+          v.w = pack_bf16(__uint_as_float(rv[d + 6]), __uint_as_float(rv[d + 7]));
+          store_swizzled_16B(tV, row, (cc >> 3) + q8, v);
+          v.x = pack_bf16(p.scale * __uint_as_float(rk[d]), p.scale * __uint_as_float(rk[d + 1]));
+          v.y = pack_bf16(p.scale * __uint_as_float(rk[d + 2]), p.scale * __uint_as_float(rk[d + 3]));
+          v.z = pack_bf16(p.scale * __uint_as_float(rk[d + 4]), p.scale * __uint_as_float(rk[d + 5]));
+          v.w = pack_bf16(p.scale * __uint_as_float(rk[d + 6]), p.scale * __uint_as_float(rk[d + 7]));
+          store_swizzled_16B(tK, row, (cc >> 3) + q8, v);
+        }
+      }
+      fence_proxy_async();
+      asm volatile("bar.sync 1, 256;" ::: "memory");      // the eight softmax warps
+      if (tid == 0) {
+        tma_store_3d(&mdv_out, tV, h * DK, k0, b);
+        tma_store_3d(&mdk_out, tK, h * DK, k0, b);
+        bulk_commit_group();
+        bulk_wait_group_read<0>();
+      }
+      if (want_db && p.bias_far > 0) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          far_pos += __shfl_xor_sync(0xffffffffu, far_pos, o);
+          far_neg += __shfl_xor_sync(0xffffffffu, far_neg, o);
+        }
+        if (lane == 0) {
+          const int gp = p.bias_far + p.Tq - 1, gn = -p.bias_far + p.Tq - 1;
+          if (far_pos != 0.f && gp < span) atomicAdd(&p.dbias_delta[(int64_t)h * span + gp], far_pos);
+          if (far_neg != 0.f && gn >= 0) atomicAdd(&p.dbias_delta[(int64_t)h * span + gn], far_neg);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (want_db && !*abort_flag) {
+    // window index w = (key row - query + tqp); distance = k0 + w - tqp
+    for (int w = tid; w < tqp + 128; w += kKvfThreads) {
+      const float v = dbias_s[w];
+      const int g = k0 + w - tqp + p.Tq - 1;
+      if (v != 0.f && g >= 0 && g < span) atomicAdd(&p.dbias_delta[(int64_t)h * span + g], v);
+    }
+  }
+  if (warp == 8) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// Kernel B: dQ[128 queries x DK] = scale * sum over 64-key tiles of dS[128 x 64] K[64 x DK], with dS read from the
+// key-major copy kernel A stored (so it is an MN-major A operand: two 64 x 64 boxes per tile).
+template <int DK>
+struct DqsLayout {
+  static constexpr int kStages = 4;
+  static constexpr int kABytes = 2 * 8192, kBBytes = 64 * DK * 2;
+  static constexpr int kStage = kABytes + kBBytes;
+  static constexpr int kBar = kStages * kStage;
+  static constexpr int kTotal = kBar + 256 + 1024;
+};
+
+template <int DK>
+__global__ void __launch_bounds__(192)
+attn_bwd_dq_ds_tc_kernel(const __grid_constant__ CUtensorMap mds, const __grid_constant__ CUtensorMap mk, TcParams p) {
+  using L = DqsLayout<DK>;
+  constexpr int NST = L::kStages;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint64_t* full = (uint64_t*)(smem + L::kBar);
+  uint64_t* empty = full + NST;
+  uint64_t* done = empty + NST;
+  uint32_t* tmem_holder = (uint32_t*)(done + 1);
+  volatile int* abort_flag = (volatile int*)(tmem_holder + 1);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * 128;
+  int n_kt = (p.Tk + 63) / 64;
+  if (p.causal) n_kt = min(n_kt, (q0 + 127) / 64 + 1);
+  constexpr uint32_t kTmemCols = DK;
+
+  if (tid == 0) {
+    for (int s = 0; s < NST; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(done, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) tmem_alloc(tmem_holder, kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+  bool ok = true;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int issued = 0;
+      for (int t = 0; t < n_kt; ++t) {
+        const int s = t % NST;
+        if (!mbar_wait(&empty[s], ((t / NST) & 1) ^ 1, abort_flag, p.status, 51)) { ok = false; break; }
+        unsigned char* sa = smem + s * L::kStage;
+        mbar_arrive_expect_tx(&full[s], L::kStage);
+        tma_load_3d(sa, &mds, q0, t * 64, b * p.H + h, &full[s]);
+        tma_load_3d(sa + 8192, &mds, q0 + 64, t * 64, b * p.H + h, &full[s]);
+#pragma unroll
+        for (int c = 0; c < DK / 64; ++c)
+          tma_load_3d(sa + L::kABytes + c * 8192, &mk, h * DK + c * 64, t * 64, b, &full[s]);
+        ++issued;
+      }
+      if (!ok && issued > 0) {   // a wait ran out: give loads still in flight a bounded time to land
+        long long t0 = clock64();
+        while (clock64() - t0 < 4000000ll) {}
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(128, DK, true, true);
+      for (int t = 0; t < n_kt; ++t) {
+        const int s = t % NST;
+        if (!mbar_wait(&full[s], (t / NST) & 1, abort_flag, p.status, 52)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t la = desc_lo_mn(smem_u32(smem + s * L::kStage)), lb = la + (L::kABytes >> 4);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          umma_bf16_lo(tmem_base, la + ((ks * 2048) >> 4), lb + ((ks * 2048) >> 4), idesc, (t | ks) != 0);
+        umma_commit(&empty[s]);
+      }
+      if (ok) umma_commit(done);
+    }
+  } else {
+    // epilogue: warps 2-5; warp w may touch tensor-memory lanes 32 (w % 4) ..
+    const int quad = warp & 3, row = quad * 32 + lane, i = q0 + row;
+    ok = mbar_wait(done, 0, abort_flag, p.status, 53);
+    if (ok) {
+      tc_fence_after();
+      bf16* drow = (bf16*)p.out0 + (int64_t)(b * p.Tq + i) * p.ld0 + h * DK;
+      const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
+#pragma unroll
+      for (int c = 0; c < DK / 32; ++c) {
+        uint32_t r[32];
+        if (n_kt > 0) {
+          tmem_ld_32x32b_x32(tmem_base + lane_off + c * 32, r);
+          tmem_wait_ld_dep(r);
+        } else {
+#pragma unroll
+          for (int d = 0; d < 32; ++d) r[d] = 0u;
+        }
+        if (i < p.Tq) {
+#pragma unroll
+          for (int d = 0; d < 32; d += 8) {
+            uint4 v;
+            v.x = pack_bf16(p.scale * __uint_as_float(r[d]), p.scale * __uint_as_float(r[d + 1]));
+            v.y = pack_bf16(p.scale * __uint_as_float(r[d + 2]), p.scale * __uint_as_float(r[d + 3]));
+            v.z = pack_bf16(p.scale * __uint_as_float(r[d + 4]), p.scale * __uint_as_float(r[d + 5]));
+            v.w = pack_bf16(p.scale * __uint_as_float(r[d + 6]), p.scale * __uint_as_float(r[d + 7]));
+            *reinterpret_cast<uint4*>(drow + c * 32 + d) = v;
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
 }
 
 // ----------------------------------------------------------------------------- host side
@@ -950,14 +1493,51 @@ cudaError_t fwd_launch(const AttnArgs& a, int* status, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+// One pass over the scores: kernel A (dK, dV, dS^T to scratch) then kernel B (dQ from the stored dS^T).
+template <int DK>
+cudaError_t bwd_fused_launch(const AttnArgs& a, int* status, cudaStream_t st) {
+  const int I = a.H * DK;
+  const int tqp = (a.Tq + 63) / 64 * 64, tkp = (a.Tk + 127) / 128 * 128;
+  TcParams p = base_params(a, status);
+  CUtensorMap mq, mdo, mk, mv, mds_st, mds_ld, mk64, mdk_out, mdv_out;
+  if (!make_map3(&mq, a.Q, I, a.Tq, a.B, a.ldq, 64) || !make_map3(&mdo, a.dO, I, a.Tq, a.B, a.lddo, 64) ||
+      !make_map3(&mk, a.K, I, a.Tk, a.B, a.ldk, 128) || !make_map3(&mv, a.V, I, a.Tk, a.B, a.ldv, 128) ||
+      !make_map3(&mk64, a.K, I, a.Tk, a.B, a.ldk, 64) ||
+      !make_map3(&mdk_out, a.dK, I, a.Tk, a.B, a.lddk, 128) || !make_map3(&mdv_out, a.dV, I, a.Tk, a.B, a.lddv, 128) ||
+      !make_map3(&mds_st, a.ds_scratch, tqp, tkp, a.B * a.H, tqp, 128) ||
+      !make_map3(&mds_ld, a.ds_scratch, tqp, tkp, a.B * a.H, tqp, 64))
+    return cudaErrorInvalidValue;
+  {
+    int smem = KvfLayout<DK>::bytes(a.Tq, a.dbias_delta != nullptr);
+    cudaError_t e = cudaFuncSetAttribute(attn_bwd_kvf_tc_kernel<DK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    dim3 grid((a.Tk + 127) / 128, a.H, a.B);
+    attn_bwd_kvf_tc_kernel<DK><<<grid, kKvfThreads, smem, st>>>(mq, mdo, mk, mv, mds_st, mdk_out, mdv_out, p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  {
+    int smem = DqsLayout<DK>::kTotal;
+    cudaError_t e = cudaFuncSetAttribute(attn_bwd_dq_ds_tc_kernel<DK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    p.out0 = a.dQ; p.ld0 = a.lddq;
+    dim3 grid((a.Tq + 127) / 128, a.H, a.B);
+    attn_bwd_dq_ds_tc_kernel<DK><<<grid, 192, smem, st>>>(mds_ld, mk64, p);
+    return cudaGetLastError();
+  }
+}
+
 template <int DK>
 cudaError_t bwd_launch(const AttnArgs& a, int* status, cudaStream_t st) {
   int I = a.H * DK;
-  int warps = a.B * a.Tq * a.H;
-  attn_delta_tc_kernel<DK><<<(warps + 7) / 8, 256, 0, st>>>((const bf16*)a.O, a.ldo, a.O32, a.ldo32,
-                                                            (const bf16*)a.dO, a.lddo, a.delta, a.B, a.H, a.Tq);
+  const int64_t dthreads = (int64_t)a.B * a.Tq * (I / 8);
+  attn_delta_tc_kernel<DK><<<(unsigned)((dthreads + 255) / 256), 256, 0, st>>>(
+      (const bf16*)a.O, a.ldo, a.O32, a.ldo32, (const bf16*)a.dO, a.lddo, a.delta, a.B, a.H, a.Tq);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
+  if constexpr (DK == 64) {
+    if (attn_tc_onepass_supported(a)) return bwd_fused_launch<DK>(a, status, st);
+  }
   TcParams p = base_params(a, status);
   {
     CUtensorMap mq, mdo, mk, mv;
@@ -990,6 +1570,17 @@ cudaError_t bwd_launch(const AttnArgs& a, int* status, cudaStream_t st) {
 }
 
 }  // namespace
+
+int64_t attn_tc_ds_scratch_bytes(int B, int H, int Tq, int Tk) {
+  int64_t tqp = (Tq + 63) / 64 * 64, tkp = (Tk + 127) / 128 * 128;
+  return (int64_t)B * H * tqp * tkp * 2;
+}
+
+bool attn_tc_onepass_supported(const AttnArgs& a) {
+  return a.dk == 64 && a.ds_scratch && ((uintptr_t)a.ds_scratch & 127) == 0 &&
+         a.ds_bytes >= attn_tc_ds_scratch_bytes(a.B, a.H, a.Tq, a.Tk) &&
+         KvfLayout<64>::bytes(a.Tq, a.dbias_delta != nullptr) <= 227 * 1024;
+}
 
 bool attn_tc_supported(const AttnArgs& a) {
   if (a.dk != 64 && a.dk != 128) return false;

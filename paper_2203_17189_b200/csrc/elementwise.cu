@@ -189,6 +189,73 @@ __global__ void rmsnorm_bwd_kernel(const TDY* __restrict__ dY, const float* __re
   for (int c = threadIdx.x; c < d; c += blockDim.x) partial[(int64_t)blockIdx.x * d + c] = s_dg[c];
 }
 
+// Same arithmetic, one row per CTA pass (d <= 1024 * NCH): thread t owns columns [4t, 4t + 4) of each 1024-column
+// chunk for every row its CTA visits, so g and the dg partial sums of those columns live in registers (no shared
+// atomics), a row's x, dy and incoming dx are each read exactly once, and all of a row's loads are in flight before
+// the one block-wide reduction it needs.
+template <typename T, typename TDY, int NCH>
+__global__ void __launch_bounds__(256)
+rmsnorm_bwd_rows_kernel(const TDY* __restrict__ dY, const float* __restrict__ X, const float* __restrict__ rstd,
+                        const T* __restrict__ g, const float* dX_in, float* dX_out, T* __restrict__ dXb,
+                        float* __restrict__ partial, int rows, int d) {
+  __shared__ float red[2][8];
+  const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+  float4 gv[NCH], acc[NCH];
+#pragma unroll
+  for (int ch = 0; ch < NCH; ++ch) {
+    const int c = ch * 1024 + tid * 4;
+    gv[ch] = c < d ? load4(g + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    acc[ch] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  const float inv_d = 1.f / (float)d;
+  int par = 0;
+  for (int row = blockIdx.x; row < rows; row += gridDim.x, par ^= 1) {
+    const int64_t off = (int64_t)row * d;
+    float4 xv[NCH], dv[NCH], pv[NCH];
+#pragma unroll
+    for (int ch = 0; ch < NCH; ++ch) {
+      const int c = ch * 1024 + tid * 4;
+      const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+      xv[ch] = c < d ? load4(X + off + c) : z;
+      dv[ch] = c < d ? load4(dY + off + c) : z;
+      pv[ch] = (c < d && dX_in != nullptr) ? load4(dX_in + off + c) : z;
+    }
+    const float r = rstd[row];
+    float m = 0.f;
+#pragma unroll
+    for (int ch = 0; ch < NCH; ++ch)
+      m += dv[ch].x * gv[ch].x * xv[ch].x + dv[ch].y * gv[ch].y * xv[ch].y + dv[ch].z * gv[ch].z * xv[ch].z +
+           dv[ch].w * gv[ch].w * xv[ch].w;
+    m = warp_sum(m);
+    if (lane == 0) red[par][w] = m;
+    __syncthreads();      // red[par] is rewritten two rows later, behind the next row's barrier
+    float tot = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) tot += red[par][i];
+    const float r3m = r * r * r * tot * inv_d;
+#pragma unroll
+    for (int ch = 0; ch < NCH; ++ch) {
+      const int c = ch * 1024 + tid * 4;
+      if (c < d) {
+        float4 o;
+        o.x = r * dv[ch].x * gv[ch].x - xv[ch].x * r3m + pv[ch].x;
+        o.y = r * dv[ch].y * gv[ch].y - xv[ch].y * r3m + pv[ch].y;
+        o.z = r * dv[ch].z * gv[ch].z - xv[ch].z * r3m + pv[ch].z;
+        o.w = r * dv[ch].w * gv[ch].w - xv[ch].w * r3m + pv[ch].w;
+        store4(dX_out + off + c, o);
+        if (dXb != nullptr) store4(dXb + off + c, o);
+        acc[ch].x += dv[ch].x * xv[ch].x * r; acc[ch].y += dv[ch].y * xv[ch].y * r;
+        acc[ch].z += dv[ch].z * xv[ch].z * r; acc[ch].w += dv[ch].w * xv[ch].w * r;
+      }
+    }
+  }
+#pragma unroll
+  for (int ch = 0; ch < NCH; ++ch) {
+    const int c = ch * 1024 + tid * 4;
+    if (c < d) store4(partial + (int64_t)blockIdx.x * d + c, acc[ch]);
+  }
+}
+
 __global__ void colsum_kernel(const float* __restrict__ partial, int n_part, int d, float* __restrict__ out) {
   // block (32, 16): 32 columns, the partial rows split over 16 groups, then a shared-memory tree
   __shared__ float red[16][33];
@@ -477,8 +544,7 @@ cudaError_t launch_rmsnorm_fwd(int dtype, const float* X, const void* g, void* Y
 }
 
 int rmsnorm_bwd_parts(int rows) {
-  int p = (rows + 7) / 8;
-  if (p > 296) p = 296;
+  int p = rows < 592 ? rows : 592;      // four resident CTAs per SM
   if (p < 1) p = 1;
   return p;
 }
@@ -487,18 +553,39 @@ cudaError_t launch_rmsnorm_bwd(int dtype, const void* dy, int dy_f32, const floa
                                const void* g, const float* dX_in, float* dX_out, void* dXb, float* dg,
                                float* partial, int rows, int d, cudaStream_t st) {
   int parts = rmsnorm_bwd_parts(rows);
-  size_t sm = (size_t)d * sizeof(float);
+  if (d <= 4096) {
+#define RBR(T, TDY, NCH)                                                                                          \
+  rmsnorm_bwd_rows_kernel<T, TDY, NCH><<<parts, 256, 0, st>>>((const TDY*)dy, X, rstd, (const T*)g, dX_in, dX_out, \
+                                                              (T*)dXb, partial, rows, d)
+#define RBR_N(T, TDY)                                                     \
+  do {                                                                    \
+    if (d <= 1024) RBR(T, TDY, 1); else if (d <= 2048) RBR(T, TDY, 2);    \
+    else RBR(T, TDY, 4);                                                  \
+  } while (0)
+    if (dtype == DT_F32) {
+      RBR_N(float, float);
+    } else if (dy_f32) {
+      RBR_N(bf16, float);
+    } else {
+      RBR_N(bf16, bf16);
+    }
+#undef RBR_N
+#undef RBR
+  } else {
+    if (parts > 296) parts = 296;
+    size_t sm = (size_t)d * sizeof(float);
 #define RB(T, TDY)                                                                                     \
   rmsnorm_bwd_kernel<T, TDY><<<parts, 256, sm, st>>>((const TDY*)dy, X, rstd, (const T*)g, dX_in, dX_out, \
                                                      (T*)dXb, partial, rows, d)
-  if (dtype == DT_F32) {
-    RB(float, float);
-  } else if (dy_f32) {
-    RB(bf16, float);
-  } else {
-    RB(bf16, bf16);
-  }
+    if (dtype == DT_F32) {
+      RB(float, float);
+    } else if (dy_f32) {
+      RB(bf16, float);
+    } else {
+      RB(bf16, bf16);
+    }
 #undef RB
+  }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   colsum_kernel<<<blocks_for(d, 32), dim3(32, 16), 0, st>>>(partial, parts, d, dg);

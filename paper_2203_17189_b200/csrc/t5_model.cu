@@ -8,6 +8,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <algorithm>
 #include <string>
 #include <vector>
 
@@ -42,6 +43,8 @@ struct Workspace {
   float *bias_enc, *bias_dec, *dbias_enc, *dbias_dec, *norm_partial, *delta;
   float *dX_enc, *dX_dec, *dY32;
   void *dXb_enc, *dXb_dec, *dh, *dhg, *dy, *dctx, *dqkv, *dkv;
+  void* ds_scratch;      // bf16 dS^T of one attention call (one-pass attention backward)
+  int64_t ds_bytes;
   int64_t bytes;
 };
 
@@ -236,6 +239,17 @@ void plan_workspace(const t5_handle* h, int B, int Te, int Td, char* base, Works
   w->dctx = take(Nmax * I * es);
   w->dqkv = take(Nmax * 3 * I * es);
   w->dkv = take(Ne * 2 * I * es);
+  w->ds_scratch = nullptr;
+  w->ds_bytes = 0;
+  if (c.dtype == DT_BF16 && c.d_kv == 64 && !(c.flags & (2 | (1 << 17)))) {
+    int64_t need = attn_tc_ds_scratch_bytes(B, (int)H, Td, Td);
+    if (encdec) {
+      need = std::max(need, attn_tc_ds_scratch_bytes(B, (int)H, Te, Te));
+      need = std::max(need, attn_tc_ds_scratch_bytes(B, (int)H, Td, Te));
+    }
+    w->ds_scratch = take(need);
+    w->ds_bytes = need;
+  }
   w->bytes = cur;
 }
 
@@ -419,6 +433,7 @@ void attn_backward(Ctx& cx, const AttnP& p, const AttnWs& a, float* dX, void* dX
   AttnArgs t;
   attn_args(cx, a, gm, cross, &t);
   t.dO = w.dctx; t.lddo = I; t.delta = w.delta; t.dbias_delta = gm.dbias; t.bias_far = gm.far;
+  t.ds_scratch = w.ds_scratch; t.ds_bytes = w.ds_bytes;
   if (cross) {
     t.dQ = w.dqkv; t.lddq = I;
     t.dK = w.dkv; t.dV = eoff(cx.h, w.dkv, I); t.lddk = t.lddv = 2 * I;
@@ -906,6 +921,40 @@ int t5_attention(int32_t dtype, int32_t impl, int32_t backward, int32_t B, int32
     if (dtype != DT_BF16 || !attn_tc_supported(a)) return T5_ERR_ARG;
     e = backward ? attn_bwd_tc(a, nullptr, st) : attn_fwd_tc(a, nullptr, st);
   }
+  return e == cudaSuccess ? T5_OK : T5_ERR_CUDA;
+}
+
+int t5_attention_ds_scratch_bytes(int32_t B, int32_t H, int32_t Tq, int32_t Tk, int64_t* bytes) {
+  if (!bytes) return T5_ERR_NULL;
+  if (B < 0 || H < 1 || Tq < 1 || Tk < 1) return T5_ERR_ARG;
+  *bytes = attn_tc_ds_scratch_bytes(B, H, Tq, Tk);
+  return T5_OK;
+}
+
+int t5_attention_backward_onepass(int32_t B, int32_t H, int32_t Tq, int32_t Tk, int32_t d_kv, int32_t causal,
+                                  float scale, const void* d_q, int32_t ldq, const void* d_k, int32_t ldk,
+                                  const void* d_v, int32_t ldv, const void* d_o, int32_t ldo, const float* d_o32,
+                                  const float* d_lse, const int32_t* d_code_q, const int32_t* d_code_k,
+                                  const float* d_bias_delta, const void* d_do, int32_t lddo, void* d_dq,
+                                  int32_t lddq, void* d_dk, int32_t lddk, void* d_dv, int32_t lddv, float* d_delta,
+                                  float* d_dbias_delta, int32_t bias_far, void* d_ds_scratch,
+                                  int64_t ds_scratch_bytes, void* stream) {
+  if (!d_q || !d_k || !d_v || !d_o || !d_lse || !d_code_q || !d_code_k || !d_do || !d_dq || !d_dk || !d_dv ||
+      !d_delta || !d_ds_scratch)
+    return T5_ERR_NULL;
+  if (B < 0 || H < 1 || Tq < 1 || Tk < 1 || d_kv != 64 || bias_far < 0) return T5_ERR_ARG;
+  if (ds_scratch_bytes < attn_tc_ds_scratch_bytes(B, H, Tq, Tk) || ((uintptr_t)d_ds_scratch & 127)) return T5_ERR_ARG;
+  AttnArgs a;
+  memset(&a, 0, sizeof a);
+  a.O32 = const_cast<float*>(d_o32); a.ldo32 = H * d_kv;
+  a.Q = d_q; a.K = d_k; a.V = d_v; a.O = const_cast<void*>(d_o); a.ldq = ldq; a.ldk = ldk; a.ldv = ldv; a.ldo = ldo;
+  a.lse = const_cast<float*>(d_lse);
+  a.B = B; a.H = H; a.Tq = Tq; a.Tk = Tk; a.dk = d_kv; a.code_q = d_code_q; a.code_k = d_code_k; a.causal = causal;
+  a.bias_delta = d_bias_delta; a.scale = scale; a.dO = d_do; a.lddo = lddo; a.dQ = d_dq; a.dK = d_dk; a.dV = d_dv;
+  a.lddq = lddq; a.lddk = lddk; a.lddv = lddv; a.delta = d_delta; a.dbias_delta = d_dbias_delta;
+  a.bias_far = bias_far; a.ds_scratch = d_ds_scratch; a.ds_bytes = ds_scratch_bytes;
+  if (!attn_tc_supported(a) || !attn_tc_onepass_supported(a)) return T5_ERR_ARG;
+  cudaError_t e = attn_bwd_tc(a, nullptr, (cudaStream_t)stream);
   return e == cudaSuccess ? T5_OK : T5_ERR_CUDA;
 }
 

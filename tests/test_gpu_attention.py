@@ -73,8 +73,12 @@ CASES = [
 ]
 
 
-@pytest.mark.parametrize("impl", [0, 1])
-@pytest.mark.parametrize("B,H,Tq,Tk,dk,causal,use_bias,mode", CASES)
+# impl 2: tcgen05 forward, then the one-pass backward entry point (dS goes through a scratch buffer)
+@pytest.mark.parametrize("impl", [0, 1, 2])
+@pytest.mark.parametrize("B,H,Tq,Tk,dk,causal,use_bias,mode", CASES + [
+    (1, 2, 640, 640, 64, True, True, "packed"),
+    (2, 2, 50, 330, 64, False, True, "pad"),
+])
 def test_attention_forward_backward(impl, B, H, Tq, Tk, dk, causal, use_bias, mode):
     rng = np.random.default_rng(B * 1000 + Tq + Tk + dk)
     I = H * dk
@@ -97,6 +101,12 @@ def test_attention_forward_backward(impl, B, H, Tq, Tk, dk, causal, use_bias, mo
         code_q = np.minimum(code_q, 1)
     bias = (rng.standard_normal((H, Tq + Tk - 1)) * 0.5).astype(np.float32) if use_bias else None
     scale = 0.25 if dk == 64 else 0.2
+    # one-pass backward with a saturated bias: constant beyond +-far, whose dS mass is then booked at +-far
+    far = 48 if (impl == 2 and use_bias and Tq >= 200) else 0
+    if far:
+        c = Tq - 1
+        bias[:, c + far:] = bias[:, c + far:c + far + 1]
+        bias[:, :c - far] = bias[:, c - far:c - far + 1]
 
     o = torch.full((B * Tq, I), float("nan"), dtype=bf, device=DEV)
     lse = torch.empty(B, H, Tq, dtype=torch.float32, device=DEV)
@@ -109,9 +119,17 @@ def test_attention_forward_backward(impl, B, H, Tq, Tk, dk, causal, use_bias, mo
     ck_d = torch.from_numpy(code_k).to(DEV)
     bias_d = None if bias is None else torch.from_numpy(bias).to(DEV)
     o32 = torch.full((B * Tq, I), float("nan"), dtype=torch.float32, device=DEV) if B != 3 else None
-    Bd.t5_attention(impl, False, B, H, Tq, Tk, dk, causal, scale, q, k, v, o, lse, cq_d, ck_d, bias_d, o32=o32)
-    Bd.t5_attention(impl, True, B, H, Tq, Tk, dk, causal, scale, q, k, v, o, lse, cq_d, ck_d, bias_d,
-                    do=do, dq=dq, dk=dk_t, dv=dv_t, delta=delta, dbias_delta=dbias, o32=o32)
+    if impl == 2 and dk != 64:
+        pytest.skip("the one-pass backward covers d_kv 64")
+    Bd.t5_attention(min(impl, 1), False, B, H, Tq, Tk, dk, causal, scale, q, k, v, o, lse, cq_d, ck_d, bias_d, o32=o32)
+    if impl == 2:
+        nbytes = Bd.t5_attention_ds_scratch_bytes(B, H, Tq, Tk)
+        scratch = torch.full((nbytes // 2,), float("nan"), dtype=bf, device=DEV)
+        Bd.t5_attention_backward_onepass(B, H, Tq, Tk, dk, causal, scale, q, k, v, o, o32, lse, cq_d, ck_d, bias_d,
+                                         do, dq, dk_t, dv_t, delta, dbias, far, scratch)
+    else:
+        Bd.t5_attention(impl, True, B, H, Tq, Tk, dk, causal, scale, q, k, v, o, lse, cq_d, ck_d, bias_d,
+                        do=do, dq=dq, dk=dk_t, dv=dv_t, delta=delta, dbias_delta=dbias, o32=o32)
     torch.cuda.synchronize()
 
     f64 = lambda t, T: t.float().cpu().numpy().astype(np.float64).reshape(B, T, I)
@@ -132,4 +150,12 @@ def test_attention_forward_backward(impl, B, H, Tq, Tk, dk, causal, use_bias, mo
         assert np.abs(g - ref).max() <= 2e-2 * np.abs(ref).max(), (name, np.abs(g - ref).max(), np.abs(ref).max())
     if use_bias:
         g = dbias.cpu().numpy()
+        if far:
+            c = Tq - 1
+            # blocks wholly beyond +-far are booked at +-far, straddling blocks at each distance: compare folded
+            for a in (rdb, g):
+                a[:, c + far] = a[:, c + far:].sum(axis=1)
+                a[:, c + far + 1:] = 0
+                a[:, c - far] = a[:, :c - far + 1].sum(axis=1)
+                a[:, :c - far] = 0
         assert np.abs(g - rdb).max() <= 2e-2 * np.abs(rdb).max()
