@@ -262,11 +262,19 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
         mx[0] = fmaxf(mx[0], sc[c][jj]); mx[1] = fmaxf(mx[1], sc[c][jj + 1]);
         mx[2] = fmaxf(mx[2], sc[c][jj + 2]); mx[3] = fmaxf(mx[3], sc[c][jj + 3]);
       }
-    const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])));
+    // The reference point m_run of a row only follows its true maximum when that has grown by more than
+    // kLazy (log2 units): until then exp2(score - m_run) <= 2^kLazy, which float32 sums and bfloat16
+    // probabilities hold as well as values below one, and the accumulator rows need no rescaling.  The result
+    // O = acc / l and lse = m_run + log2(l) do not depend on which reference point was used.
+    constexpr float kLazy = 8.f;
+    const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+    const bool grow = m_tile > m_run + kLazy || (m_run == -INFINITY && m_tile != -INFINITY);
+    const bool warp_moves = __any_sync(0xffffffffu, grow);
+    const float m_new = warp_moves ? fmaxf(m_run, m_tile) : m_run;      // a warp that rescales moves all its rows
     const float m_eff = m_new == -INFINITY ? 0.f : m_new;      // a row with no valid key so far: exp2(-inf - 0) = 0
     const float corr = ex2_approx(m_run - m_eff);
-    // rescale the accumulator rows of this warp if any of their maxima moved
-    if (t > 0 && __any_sync(0xffffffffu, m_new != m_run)) {
+    // rescale the accumulator rows of this warp if any of their reference points moved
+    if (t > 0 && warp_moves) {
 #pragma unroll
       for (int c = 0; c < DK / 32; ++c) {
         uint32_t r[32];
@@ -1145,12 +1153,14 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
     const float sc2 = p.scale * kLog2e;
     const bool has_bias = p.bias_delta != nullptr;
     float far_pos = 0.f, far_neg = 0.f;
+    // `ok` is kept warp-uniform (every wait's answer goes through a vote): the warp-level barriers below are
+    // reached by all 32 lanes or by none
     unsigned char* tP = smem + L::kP0;
     unsigned char* tD = smem + L::kDS0;
     for (int i = 0; i < n && ok; ++i) {
       const int qb = (t_begin + i) * 64;
       const uint32_t par = i & 1;
-      ok = mbar_wait_relaxed(&bars->s_full, par, abort_flag, p.status, 46);
+      ok = __all_sync(0xffffffffu, mbar_wait_relaxed(&bars->s_full, par, abort_flag, p.status, 46));
       if (!ok) break;
       tc_fence_after();
 #pragma unroll
@@ -1231,7 +1241,7 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
         }
         if (c == 0) {
           // the tile buffers are free once the accumulating MMAs of tile i-1 are done and its dS store has read them
-          ok = mbar_wait_relaxed(&bars->p_free, par ^ 1, abort_flag, p.status, 47);
+          ok = __all_sync(0xffffffffu, mbar_wait_relaxed(&bars->p_free, par ^ 1, abort_flag, p.status, 47));
         }
         if (ok) {
 #pragma unroll
@@ -1256,9 +1266,9 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->p_full);
     }
-    if (ok && n > 0) ok = mbar_wait_relaxed(&bars->acc, 0, abort_flag, p.status, 48);
+    if (n > 0) ok = __all_sync(0xffffffffu, ok && mbar_wait_relaxed(&bars->acc, 0, abort_flag, p.status, 48));
     // the last dS store must have read its tile before the tile buffers are reused for the output rows
-    if (ok && n > 0) ok = mbar_wait_relaxed(&bars->p_free, (n - 1) & 1, abort_flag, p.status, 50);
+    if (n > 0) ok = __all_sync(0xffffffffu, ok && mbar_wait_relaxed(&bars->p_free, (n - 1) & 1, abort_flag, p.status, 50));
     // every softmax thread gets here whatever happened; behind this barrier the abort flag gives the whole group
     // one answer, so the barrier inside the epilogue is reached by all of them or by none
     asm volatile("bar.sync 1, 256;" ::: "memory");
