@@ -219,7 +219,7 @@ T5_API int t5_attention(int32_t dtype, int32_t impl, int32_t backward, int32_t B
                         float* d_dbias_delta, void* stream);
 
 /* Attention backward in one pass over the scores (tcgen05 kernels, bfloat16,
- * d_kv 64): the same result as t5_attention(..., backward = 1, ...) - whose two
+ * d_kv 64 or 128): the same result as t5_attention(..., backward = 1, ...) - whose two
  * kernels each recompute the scores and the probabilities - from one kernel that
  * produces dK, dV and a bfloat16 copy of dS^T in d_ds_scratch, and a second that
  * takes dQ = scale dS K from that copy.  (Backward of the attention the
@@ -229,7 +229,7 @@ T5_API int t5_attention(int32_t dtype, int32_t impl, int32_t backward, int32_t B
  * F such that the bias is constant for (j - i) >= F and for (j - i) <= -F; the
  * dS mass of those regions is then added to the entries at +F and -F of
  * d_dbias_delta.  Other arguments as in t5_attention.  T5_ERR_ARG if the shape is
- * not covered (d_kv != 64, or a query length whose per-CTA tables exceed shared
+ * not covered (d_kv not 64 or 128, or a query length whose per-CTA tables exceed shared
  * memory) or the scratch is too small. */
 T5_API int t5_attention_ds_scratch_bytes(int32_t B, int32_t H, int32_t Tq, int32_t Tk, int64_t* bytes);
 T5_API int t5_attention_backward_onepass(

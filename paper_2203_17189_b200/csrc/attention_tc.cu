@@ -977,12 +977,11 @@ constexpr int kKvfThreads = 10 * 32;
 constexpr int kKvfSoftmaxThreads = 8 * 32;
 
 template <int DK>
-__global__ void __launch_bounds__(kKvfThreads, 2)
+__global__ void __launch_bounds__(kKvfThreads, DK == 64 ? 2 : 1)
 attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mdo,
                        const __grid_constant__ CUtensorMap mk, const __grid_constant__ CUtensorMap mv,
                        const __grid_constant__ CUtensorMap mds, const __grid_constant__ CUtensorMap mdk_out,
                        const __grid_constant__ CUtensorMap mdv_out, TcParams p) {
-  static_assert(DK == 64, "the output tiles are staged as one 128-byte-wide tile per tensor");
   using L = KvfLayout<DK>;
   constexpr int NST = L::kStages;
   extern __shared__ unsigned char smem_raw[];
@@ -1002,7 +1001,7 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
   const int n_qt = (p.Tq + 63) / 64;
   const int t_begin = p.causal ? k0 / 64 : 0;          // queries before k0 see none of these keys
   const int n = n_qt - t_begin;                        // tiles this CTA walks
-  constexpr uint32_t kTmemCols = 256;
+  constexpr uint32_t kTmemCols = DK == 64 ? 256 : 512;
   constexpr uint32_t kColS = 0, kColDP = 64, kColDV = 128, kColDK = 128 + DK;
 
   auto load_qd = [&](int i) {
@@ -1275,17 +1274,19 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
     ok = *abort_flag == 0;
     if (ok) {
       tc_fence_after();
-      // dV and dK rows go through the (now idle) P^T / dS^T tiles as 128-byte-swizzled [128 keys x 64] bf16 tiles
-      // and leave with one TMA store each: full 128-byte row segments, rows beyond Tk clipped by the tensor map
+      // dV and dK rows go through idle operand tiles as 128-byte-swizzled [128 keys x 64] bf16 tiles (one per 64
+      // columns) and leave with one TMA store per tile: full 128-byte row segments, rows beyond Tk clipped by the
+      // tensor map.  dV uses the P^T / dS^T tiles, dK the dS^T tile (d_kv 64) or the Q / dO ring (d_kv 128).
       unsigned char* tV = smem + L::kP0;
-      unsigned char* tK = smem + L::kDS0;
+      unsigned char* tK = DK == 64 ? smem + L::kDS0 : smem + L::kQD0;
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        const int cc = half * 32 + c * 16;
+      for (int c = 0; c < DK / 32; ++c) {
+        const int col = half * (DK / 2) + c * 16;          // this pass's 16 output columns
+        const int chunk = col >> 6, piece0 = (col & 63) >> 3;
         uint32_t rv[16], rk[16];
         if (n > 0) {
-          tmem_ld_32x32b_x16(tmem_base + lane_off + kColDV + cc, rv);
-          tmem_ld_32x32b_x16(tmem_base + lane_off + kColDK + cc, rk);
+          tmem_ld_32x32b_x16(tmem_base + lane_off + kColDV + col, rv);
+          tmem_ld_32x32b_x16(tmem_base + lane_off + kColDK + col, rk);
           tmem_wait_ld_dep16(rv);
           tmem_wait_ld_dep16(rk);
         } else {
@@ -1300,19 +1301,22 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
           v.y = pack_bf16(__uint_as_float(rv[d + 2]), __uint_as_float(rv[d + 3]));
           v.z = pack_bf16(__uint_as_float(rv[d + 4]), __uint_as_float(rv[d + 5]));
           v.w = pack_bf16(__uint_as_float(rv[d + 6]), __uint_as_float(rv[d + 7]));
-          store_swizzled_16B(tV, row, (cc >> 3) + q8, v);
+          store_swizzled_16B(tV + chunk * 16384, row, piece0 + q8, v);
           v.x = pack_bf16(p.scale * __uint_as_float(rk[d]), p.scale * __uint_as_float(rk[d + 1]));
           v.y = pack_bf16(p.scale * __uint_as_float(rk[d + 2]), p.scale * __uint_as_float(rk[d + 3]));
           v.z = pack_bf16(p.scale * __uint_as_float(rk[d + 4]), p.scale * __uint_as_float(rk[d + 5]));
           v.w = pack_bf16(p.scale * __uint_as_float(rk[d + 6]), p.scale * __uint_as_float(rk[d + 7]));
-          store_swizzled_16B(tK, row, (cc >> 3) + q8, v);
+          store_swizzled_16B(tK + chunk * 16384, row, piece0 + q8, v);
         }
       }
       fence_proxy_async();
       asm volatile("bar.sync 1, 256;" ::: "memory");      // the eight softmax warps
       if (tid == 0) {
-        tma_store_3d(&mdv_out, tV, h * DK, k0, b);
-        tma_store_3d(&mdk_out, tK, h * DK, k0, b);
+#pragma unroll
+        for (int c = 0; c < DK / 64; ++c) {
+          tma_store_3d(&mdv_out, tV + c * 16384, h * DK + c * 64, k0, b);
+          tma_store_3d(&mdk_out, tK + c * 16384, h * DK + c * 64, k0, b);
+        }
         bulk_commit_group();
         bulk_wait_group_read<0>();
       }
@@ -1545,9 +1549,7 @@ cudaError_t bwd_launch(const AttnArgs& a, int* status, cudaStream_t st) {
       (const bf16*)a.O, a.ldo, a.O32, a.ldo32, (const bf16*)a.dO, a.lddo, a.delta, a.B, a.H, a.Tq);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  if constexpr (DK == 64) {
-    if (attn_tc_onepass_supported(a)) return bwd_fused_launch<DK>(a, status, st);
-  }
+  if (attn_tc_onepass_supported(a)) return bwd_fused_launch<DK>(a, status, st);
   TcParams p = base_params(a, status);
   {
     CUtensorMap mq, mdo, mk, mv;
@@ -1587,9 +1589,11 @@ int64_t attn_tc_ds_scratch_bytes(int B, int H, int Tq, int Tk) {
 }
 
 bool attn_tc_onepass_supported(const AttnArgs& a) {
-  return a.dk == 64 && a.ds_scratch && ((uintptr_t)a.ds_scratch & 127) == 0 &&
-         a.ds_bytes >= attn_tc_ds_scratch_bytes(a.B, a.H, a.Tq, a.Tk) &&
-         KvfLayout<64>::bytes(a.Tq, a.dbias_delta != nullptr) <= 227 * 1024;
+  if ((a.dk != 64 && a.dk != 128) || !a.ds_scratch || ((uintptr_t)a.ds_scratch & 127) != 0 ||
+      a.ds_bytes < attn_tc_ds_scratch_bytes(a.B, a.H, a.Tq, a.Tk))
+    return false;
+  const bool db = a.dbias_delta != nullptr;
+  return (a.dk == 64 ? KvfLayout<64>::bytes(a.Tq, db) : KvfLayout<128>::bytes(a.Tq, db)) <= 227 * 1024;
 }
 
 bool attn_tc_supported(const AttnArgs& a) {

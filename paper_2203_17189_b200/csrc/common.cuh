@@ -103,7 +103,7 @@ struct AttnArgs {
   int bias_far;             // 0, or a distance F such that the bias is constant for (j - i) >= F and constant for
                             // (j - i) <= -F (the saturated buckets): the backward may then add the whole dS mass
                             // of such regions to the entries at +F / -F instead of to each distance
-  // optional scratch of attn_tc_ds_scratch_bytes(B, H, Tq, Tk) bytes: with it the tcgen05 backward (d_kv 64) makes
+  // optional scratch of attn_tc_ds_scratch_bytes(B, H, Tq, Tk) bytes: with it the tcgen05 backward makes
   // one pass over the scores (dK, dV and a bf16 copy of dS^T in this buffer) and takes dQ from the stored dS
   void* ds_scratch = nullptr;
   int64_t ds_bytes = 0;

@@ -241,7 +241,7 @@ void plan_workspace(const t5_handle* h, int B, int Te, int Td, char* base, Works
   w->dkv = take(Ne * 2 * I * es);
   w->ds_scratch = nullptr;
   w->ds_bytes = 0;
-  if (c.dtype == DT_BF16 && c.d_kv == 64 && !(c.flags & (2 | (1 << 17)))) {
+  if (c.dtype == DT_BF16 && (c.d_kv == 64 || c.d_kv == 128) && !(c.flags & (2 | (1 << 17)))) {
     int64_t need = attn_tc_ds_scratch_bytes(B, (int)H, Td, Td);
     if (encdec) {
       need = std::max(need, attn_tc_ds_scratch_bytes(B, (int)H, Te, Te));
@@ -942,7 +942,7 @@ int t5_attention_backward_onepass(int32_t B, int32_t H, int32_t Tq, int32_t Tk, 
   if (!d_q || !d_k || !d_v || !d_o || !d_lse || !d_code_q || !d_code_k || !d_do || !d_dq || !d_dk || !d_dv ||
       !d_delta || !d_ds_scratch)
     return T5_ERR_NULL;
-  if (B < 0 || H < 1 || Tq < 1 || Tk < 1 || d_kv != 64 || bias_far < 0) return T5_ERR_ARG;
+  if (B < 0 || H < 1 || Tq < 1 || Tk < 1 || (d_kv != 64 && d_kv != 128) || bias_far < 0) return T5_ERR_ARG;
   if (ds_scratch_bytes < attn_tc_ds_scratch_bytes(B, H, Tq, Tk) || ((uintptr_t)d_ds_scratch & 127)) return T5_ERR_ARG;
   AttnArgs a;
   memset(&a, 0, sizeof a);
