@@ -61,15 +61,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
-// Common position code of n consecutive keys/queries (n = 128: one int4 per lane, n = 64: one int2),
-// or -1 if they differ.  A tile whose code equals every row's code (and lies on the allowed side of the
-// diagonal) needs no per-element mask.
-__device__ __forceinline__ int tile_code128(const int* codes, int lane) {
-  int4 c = *reinterpret_cast<const int4*>(codes + lane * 4);
-  int first = __shfl_sync(0xffffffffu, c.x, 0);
-  bool same = c.x == first && c.y == first && c.z == first && c.w == first;
-  return __all_sync(0xffffffffu, same) ? first : -1;
-}
+// Common position code of 64 consecutive keys/queries (one int2 per lane), or -1 if they differ.  A tile
+// whose code equals every row's code (and lies on the allowed side of the diagonal) needs no per-element mask.
 __device__ __forceinline__ int tile_code64(const int* codes, int lane) {
   int2 c = *reinterpret_cast<const int2*>(codes + lane * 2);
   int first = __shfl_sync(0xffffffffu, c.x, 0);

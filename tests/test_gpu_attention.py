@@ -78,10 +78,14 @@ CASES = [
 @pytest.mark.parametrize("B,H,Tq,Tk,dk,causal,use_bias,mode", CASES + [
     (1, 2, 640, 640, 64, True, True, "packed"),
     (2, 2, 50, 330, 64, False, True, "pad"),
+    # large scores (scale 1): row maxima move by more than the forward kernel's lazy-rescale threshold between tiles
+    (1, 2, 448, 448, 64, False, True, "full_hot"),
 ])
 def test_attention_forward_backward(impl, B, H, Tq, Tk, dk, causal, use_bias, mode):
     rng = np.random.default_rng(B * 1000 + Tq + Tk + dk)
     I = H * dk
+    hot = mode.endswith("_hot")
+    mode = mode[:-4] if hot else mode
     bf = torch.bfloat16
 
     def rnd(*shape, s=1.0):
@@ -100,7 +104,7 @@ def test_attention_forward_backward(impl, B, H, Tq, Tk, dk, causal, use_bias, mo
     if mode == "packed" and Tq != Tk:
         code_q = np.minimum(code_q, 1)
     bias = (rng.standard_normal((H, Tq + Tk - 1)) * 0.5).astype(np.float32) if use_bias else None
-    scale = 0.25 if dk == 64 else 0.2
+    scale = 1.0 if hot else (0.25 if dk == 64 else 0.2)
     # one-pass backward with a saturated bias: constant beyond +-far, whose dS mass is then booked at +-far
     far = 48 if (impl == 2 and use_bias and Tq >= 200) else 0
     if far:
