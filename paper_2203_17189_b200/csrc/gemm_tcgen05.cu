@@ -101,9 +101,10 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
 // Epilogue of one 128-row x BN-column accumulator tile for one warp (rows quad*32 .. +31 of the tile).
 // Each thread holds one accumulator row; going through a per-warp shared-memory tile turns the stores (and the
 // loads of the float32 addend) into 128-byte row segments instead of 32 scattered pieces.
+// Chunks (32 columns each) [c_begin, c_end) of the tile are this warp's share.
 template <int BN>
 __device__ __forceinline__ void store_tile(const Params& p, float* tbuf, uint32_t tacc, int m0, int n0, int quad,
-                                           int lane, bool add_atomic) {
+                                           int lane, bool add_atomic, int c_begin = 0, int c_end = BN / 32) {
   const int rr0 = lane >> 3, cc = (lane & 7) * 4;
   // float32 addend (residual input, or D itself when accumulating), fetched one chunk ahead of its use
   const float* addend = (!p.out_f32 || add_atomic) ? nullptr
@@ -119,9 +120,9 @@ __device__ __forceinline__ void store_tile(const Params& p, float* tbuf, uint32_
                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
     }
   };
-  fetch_addend(0, add_next);
+  fetch_addend(c_begin, add_next);
 #pragma unroll 1
-  for (int c = 0; c < BN / 32; ++c) {
+  for (int c = c_begin; c < c_end; ++c) {
     const int col0 = n0 + c * 32;
     if (col0 >= p.N) break;               // uniform across the warp
     float4 add_cur[8];
@@ -136,7 +137,7 @@ __device__ __forceinline__ void store_tile(const Params& p, float* tbuf, uint32_
           make_float4(p.alpha * __uint_as_float(r[4 * j]), p.alpha * __uint_as_float(r[4 * j + 1]),
                       p.alpha * __uint_as_float(r[4 * j + 2]), p.alpha * __uint_as_float(r[4 * j + 3]));
     __syncwarp();
-    if (addend && c + 1 < BN / 32) fetch_addend(c + 1, add_next);     // in flight while this chunk is stored
+    if (addend && c + 1 < c_end) fetch_addend(c + 1, add_next);       // in flight while this chunk is stored
     const int col = col0 + cc;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -200,12 +201,12 @@ __device__ __forceinline__ void transpose_chunk(float* tbuf, int lane, const uin
 }
 // forward: accumulator columns [0,128) = a, [128,256) = b of feature block tn; writes h = [a | b] and hg = gelu(a) b
 __device__ __forceinline__ void store_tile_geglu_fwd(const Params& p, float* tbuf, uint32_t tacc, int m0, int tn, int quad,
-                                                     int lane) {
+                                                     int lane, int c_begin = 0, int c_end = 4) {
   const int rr0 = lane >> 3, cc = (lane & 7) * 4;
   bf16* H = (bf16*)p.D;
   bf16* HG = (bf16*)p.aux;
 #pragma unroll 1
-  for (int c = 0; c < 4; ++c) {
+  for (int c = c_begin; c < c_end; ++c) {
     uint32_t ra[32], rb[32];
     tmem_ld_32x32b_x32(tacc + c * 32, ra);
     tmem_ld_32x32b_x32(tacc + 128 + c * 32, rb);
@@ -235,12 +236,12 @@ __device__ __forceinline__ void store_tile_geglu_fwd(const Params& p, float* tbu
 // backward: the accumulator is d(hg); aux = h = [a | b]; writes dh = [d(hg) b gelu'(a) | d(hg) gelu(a)]
 template <int BN>
 __device__ __forceinline__ void store_tile_geglu_bwd(const Params& p, float* tbuf, uint32_t tacc, int m0, int n0, int quad,
-                                                     int lane) {
+                                                     int lane, int c_begin = 0, int c_end = BN / 32) {
   const int rr0 = lane >> 3, cc = (lane & 7) * 4;
   const bf16* Hh = (const bf16*)p.aux;
   bf16* DH = (bf16*)p.D;
 #pragma unroll 1
-  for (int c = 0; c < BN / 32; ++c) {
+  for (int c = c_begin; c < c_end; ++c) {
     if (n0 + c * 32 >= p.N) break;
     uint32_t r[32];
     tmem_ld_32x32b_x32(tacc + c * 32, r);
@@ -459,19 +460,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // A cluster of two CTAs computes one 256 x 256 tile: CTA r loads rows [128 r, 128 r + 128) of A and of the B tile
 // into its own shared memory (plain TMA, completion counted on the leader's barrier), the leader's MMA thread issues
 // tcgen05.mma.cta_group::2 (M = 256, N = 256), each CTA's tensor memory receives its 128 rows of the result and each
-// CTA runs the epilogue of its half.  Per CTA a K slice costs 32 KB of loads instead of 48 KB, and six stages fit.
-constexpr int STAGES2 = 6;
+// CTA runs the epilogue of its half.  Per CTA a K slice costs 32 KB of loads instead of 48 KB.
+// Twelve warps: producer, MMA issuer, tensor-memory owner, one idle, and EIGHT epilogue warps - two per tensor-memory
+// lane quarter, each with half of the tile's columns.  With four, every epilogue warp sat alone on its scheduler and
+// the heavier epilogues (gated-GELU backward, float32 residual) ran at the pace of one warp's instruction latencies,
+// longer than the tile's MMAs; a second warp per scheduler hides them.  The transpose buffers of the extra warps
+// take the room of the sixth stage.
+constexpr int kThreads2 = 384;
+constexpr int STAGES2 = 5;
 struct Smem2 {
   static constexpr int kABytes = 128 * BK * 2, kBBytes = 128 * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kBarOffset = STAGES2 * kStageBytes;
   static constexpr int kEpiOffset = kBarOffset + 256;
-  static constexpr int kEpiBytes = 4 * 32 * 36 * 4;
+  static constexpr int kEpiBytes = 8 * 32 * 36 * 4;
   static constexpr int kTotal = kEpiOffset + kEpiBytes + 1024;
 };
 
 template <bool A_MN, bool B_MN>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, Params p) {
   using S = Smem2;
   constexpr int BN = 256;
@@ -495,7 +502,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES2; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 8); }   // 4 warps of each CTA
+    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 16); }  // 8 warps of each CTA
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -577,7 +584,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
-    const int quad = warp & 3;
+    const int quad = warp & 3, ew = warp - 4, ch = ew >> 2;      // ch: which half of the tile's columns
     int it = 0;
     bool ok = true;
     WorkIter wi(p, k_blocks, pair, n_pairs);
@@ -590,10 +597,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const uint32_t aph = (it >> 1) & 1;
       ok = mbar_wait(&tfull[ab], aph, abort_flag, p.status, 9);
       if (ok && w.kind == 2) {
-        // an earlier K-segment of a split tile: the storing pair (8 epilogue warps) must be done first
+        // an earlier K-segment of a split tile: the storing pair (16 epilogue warps) must be done first
         volatile int* flag = p.sk_flags + w.flag;
         long long t0 = clock64();
-        while (*flag < 8) {
+        while (*flag < 16) {
           if (clock64() - t0 > kWaitCycles) {
             if (p.status) atomicCAS(p.status, 0, 10);
             ok = false;
@@ -606,11 +613,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      float* tb = reinterpret_cast<float*>(smem + S::kEpiOffset) + quad * (32 * 36);
+      float* tb = reinterpret_cast<float*>(smem + S::kEpiOffset) + ew * (32 * 36);
       const uint32_t tacc = tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16);
-      if (p.epi == 1) store_tile_geglu_fwd(p, tb, tacc, m0, tn, quad, lane);
-      else if (p.epi == 2) store_tile_geglu_bwd<BN>(p, tb, tacc, m0, n0, quad, lane);
-      else store_tile<BN>(p, tb, tacc, m0, n0, quad, lane, w.kind == 2);
+      if (p.epi == 1) store_tile_geglu_fwd(p, tb, tacc, m0, tn, quad, lane, ch * 2, ch * 2 + 2);
+      else if (p.epi == 2) store_tile_geglu_bwd<BN>(p, tb, tacc, m0, n0, quad, lane, ch * 4, ch * 4 + 4);
+      else store_tile<BN>(p, tb, tacc, m0, n0, quad, lane, w.kind == 2, ch * 4, ch * 4 + 4);
       if (w.kind == 1) {
         __threadfence();
         __syncwarp();
@@ -718,7 +725,7 @@ cudaError_t launch2(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap&
   } else if (tiles < pairs) {
     pairs = tiles;
   }
-  kern<<<2 * pairs, kThreads, Smem2::kTotal, st>>>(ma, mb, p);
+  kern<<<2 * pairs, kThreads2, Smem2::kTotal, st>>>(ma, mb, p);
   return cudaGetLastError();
 }
 
