@@ -205,6 +205,8 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=1)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--flags", type=int, default=0)
+    ap.add_argument("--recompute", type=int, default=0, choices=[0, 1],
+                    help="activation policy (0 keeps everything; the reported number uses 0)")
     args = ap.parse_args()
     cfg = WL.model_dims(args.workload)
     if args.batch:
@@ -234,7 +236,7 @@ def main():
 
     Bd.lib()   # fails loudly if the CUDA library is missing
     B, Te, Td = cfg["batch"], cfg["enc_len"], cfg["dec_len"]
-    h = Bd.Handle(Bd.make_config(cfg, B, Te, Td, cfg["dtype"], flags=args.flags))
+    h = Bd.Handle(Bd.make_config(cfg, B, Te, Td, cfg["dtype"], flags=args.flags, recompute=args.recompute))
     n = h.t5_param_count()
     params = torch.empty(n, dtype=h.torch_dtype, device=dev)
     h.t5_init_params(params, 1234 + rank, 0.02)
@@ -327,7 +329,8 @@ def main():
         "config": {"workload": args.workload, "layers": [cfg["n_enc_layers"], cfg["n_dec_layers"]], "batch_rows": B, "enc_len": Te, "dec_len": Td,
                    "tokens_per_step": tokens_per_step, "nonpad_tokens_per_step": nonpad,
                    "l2": f"working set {ws_bytes / 1e9:.1f} GB of activations >> 126 MB L2; no explicit flush",
-                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "activation_recomputation": bool(args.recompute)},
         "mfu": {"step_tflop": flops / 1e12, "achieved_tflops": flops / sec / 1e12,
                 "vs_nominal_2250": flops / sec / 1e12 / NOMINAL_BF16_TFLOPS,
                 "vs_measured_burst": flops / sec / 1e12 / float(peaks.get("bf16_tflops", 1590.0)),

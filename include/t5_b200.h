@@ -67,8 +67,11 @@ typedef struct {
   float z_loss, rms_eps, attn_scale, logit_scale; /* 1e-4, 1e-6, 1.0, d_model^-1/2 */
   int32_t dtype;            /* 0: float32 everywhere (validation mode);
                                1: bfloat16 parameters/operands, float32 accumulation */
-  int32_t recompute;        /* activation policy: 0 keep everything, 1 recompute cheap
-                               element-wise pieces in the backward pass */
+  int32_t recompute;        /* activation policy: 0 keep everything; 1 do not keep the normed
+                               activations and the gated-GELU product of each sub-layer but
+                               recompute them (one RMSNorm pass, one gated-GELU pass) in the
+                               backward pass right before the weight-gradient GEMMs that read
+                               them: a smaller workspace for a few per cent of step time */
   int32_t flags;            /* debugging aids for bfloat16 mode: bit 0 = use the plain SIMT
                                GEMM kernel, bit 1 = use the plain SIMT attention kernels,
                                bit 2 = do NOT run the GEMMs on CTA pairs (cta_group::2),

@@ -172,10 +172,16 @@ void plan_workspace(const t5_handle* h, int B, int Te, int Td, char* base, Works
   if (!encdec) Te = 0;
   int64_t Ne = (int64_t)B * Te, Nd = (int64_t)B * Td, Nmax = Ne > Nd ? Ne : Nd;
   int Tmax = Te > Td ? Te : Td;
+  // Activation policy 1: the normed activations y and the gated product hg are not kept per sub-layer; the
+  // forward pass writes them into one shared buffer each (the next GEMM consumes them at once) and the backward
+  // pass recomputes them from the saved x (and rstd) / pre-activations h right before the weight-gradient GEMMs.
+  const bool recompute = c.recompute == 1;
+  void* shared_y = nullptr;      // taken below, behind the status word
+  void* shared_hg = nullptr;
   auto attn_ws = [&](int64_t Nq, int64_t Nk, int Tq, bool cross) {
     AttnWs a;
     a.x = (float*)take(Nq * d * 4);
-    a.y = take(Nq * d * es);
+    a.y = recompute ? shared_y : take(Nq * d * es);
     a.rstd = (float*)take(Nq * 4);
     a.q = take(Nq * (cross ? I : 3 * I) * es);
     a.kv = cross ? take(Nk * 2 * I * es) : nullptr;
@@ -187,14 +193,18 @@ void plan_workspace(const t5_handle* h, int B, int Te, int Td, char* base, Works
   auto ffn_ws = [&](int64_t N) {
     FfnWs f;
     f.x = (float*)take(N * d * 4);
-    f.y = take(N * d * es);
+    f.y = recompute ? shared_y : take(N * d * es);
     f.rstd = (float*)take(N * 4);
     f.h = take(N * 2 * F * es);
-    f.hg = take(N * F * es);
+    f.hg = recompute ? shared_hg : take(N * F * es);
     return f;
   };
   w->status = (int*)take(4);          // first, so its address does not depend on the batch shape
   w->sk_flags = (int*)take((int64_t)kSkSlices * kSkSliceInts * 4);   // per-GEMM flag slices of the stream-K tails
+  if (recompute) {
+    shared_y = take(Nmax * d * es);
+    shared_hg = take(Nmax * F * es);
+  }
   w->enc_attn.clear(); w->enc_ffn.clear(); w->dec_self.clear(); w->dec_cross.clear(); w->dec_ffn.clear();
   if (encdec) {
     for (int l = 0; l < c.n_enc_layers; ++l) {
@@ -447,6 +457,11 @@ void attn_backward(Ctx& cx, const AttnP& p, const AttnWs& a, float* dX, void* dX
     CKL(CAT_ATTN_BWD, 3, attn_bwd_simt(dt, t, cx.st), "attn_bwd");
   dbg_round(cx, w.dqkv, (int64_t)Nq * (cross ? I : 3 * I), RB_DQKV);
   if (cross) dbg_round(cx, w.dkv, (int64_t)Nk * 2 * I, RB_DQKV);
+  if (c.recompute == 1) {
+    CKL(CAT_NORM, 1, launch_rmsnorm_fwd(dt, a.x, pptr(cx.h, cx.params, p.norm), a.y, a.rstd, Nq, d, c.rms_eps, cx.st),
+       "rmsnorm_fwd (recomputed)");
+    dbg_round(cx, a.y, (int64_t)Nq * d, RB_Y);
+  }
   if (!cross) {
     proj_wgrad(cx, w.dqkv, 3 * I, a.y, d, p.q, Nq, 3 * I, d, 1.f, "wgrad qkv");
     proj_dgrad(cx, w.dqkv, 3 * I, p.q, Nq, 3 * I, d, w.dy, d, 1.f, 0, 0, "dgrad qkv");
@@ -500,6 +515,10 @@ void ffn_backward(Ctx& cx, const FfnP& p, const FfnWs& f, float* dX, void* dXb, 
   const t5_config& c = cx.h->cfg;
   Workspace& w = *cx.w;
   int d = c.d_model, F = c.d_ff, dt = c.dtype, n = (int)N;
+  if (c.recompute == 1) {
+    CKL(CAT_GEGLU, 1, launch_geglu_fwd(dt, f.h, f.hg, n, F, cx.st), "geglu_fwd (recomputed)");
+    dbg_round(cx, f.hg, N * F, RB_HG);
+  }
   proj_wgrad(cx, dXb, d, f.hg, F, p.wo, n, d, F, 1.f, "wgrad ffn.wo");
   GemmArgs gb{};
   gb.M = n; gb.N = F; gb.K = d; gb.alpha = 1.f;
@@ -513,6 +532,11 @@ void ffn_backward(Ctx& cx, const FfnP& p, const FfnWs& f, float* dX, void* dXb, 
     dbg_round(cx, w.dhg, N * F, RB_DHG);
     CKL(CAT_GEGLU, 1, launch_geglu_bwd(dt, w.dhg, f.h, w.dh, n, F, cx.st), "geglu_bwd");
     dbg_round(cx, w.dh, N * 2 * F, RB_DH);
+  }
+  if (c.recompute == 1) {
+    CKL(CAT_NORM, 1, launch_rmsnorm_fwd(dt, f.x, pptr(cx.h, cx.params, p.norm), f.y, f.rstd, n, d, c.rms_eps, cx.st),
+       "rmsnorm_fwd (recomputed)");
+    dbg_round(cx, f.y, N * d, RB_Y);
   }
   proj_wgrad(cx, w.dh, 2 * F, f.y, d, p.wi0, n, 2 * F, d, 1.f, "wgrad ffn.wi");
   proj_dgrad(cx, w.dh, 2 * F, p.wi0, n, 2 * F, d, w.dy, d, 1.f, 0, 0, "dgrad ffn.wi");

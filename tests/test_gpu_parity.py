@@ -55,7 +55,7 @@ class Runner:
         return self.loss4.cpu().numpy().astype(np.float64), self.grads.cpu().numpy()
 
 
-def check_step(dims, batch, dtype, flags=0, seed=11, stddev=None, tol=None, table_out=None, floor=False):
+def check_step(dims, batch, dtype, flags=0, seed=11, stddev=None, tol=None, table_out=None, floor=False, recompute=0):
     """One step on the GPU against the float64 oracle.
 
     tol = (min cosine, max error / max|ref|) per gradient tensor; default: the
@@ -69,7 +69,7 @@ def check_step(dims, batch, dtype, flags=0, seed=11, stddev=None, tol=None, tabl
         stddev = 0.05 if dtype == "f32" else 0.02     # bf16 workloads use the N(0, 0.02) recipe
     B, Td = batch["dec_targets"].shape
     Te = 0 if batch["enc_tokens"] is None else batch["enc_tokens"].shape[1]
-    r = Runner(dims, B, Te, Td, dtype, flags=flags)
+    r = Runner(dims, B, Te, Td, dtype, flags=flags, recompute=recompute)
     shapes = PR.oracle_shapes_from_manifest(r.man)
     named = WL.make_params(shapes, seed, stddev=stddev, scale_jitter=0.05)
     named = r.set_params(named)
@@ -244,6 +244,23 @@ def test_step_large_widths(name, dtype):
         check_step(dims, batch, "f32", stddev=0.02, tol=(0.999999, 5e-4))
     else:
         check_step(dims, batch, "bf16", floor=True)
+
+
+def test_step_activation_recomputation():
+    """Activation policy 1 (normed activations and gated product recomputed in the backward pass): same bars
+    against the oracle as policy 0, and a smaller workspace.  The XL-width case runs the gated GELU inside the
+    GEMM epilogue in the forward pass and the separate kernel for the recomputation."""
+    dims = WL.model_dims("tiny")
+    batch = WL.make_batch("tiny")
+    r1, _, loss1, _ = check_step(dims, batch, "f32", stddev=0.02, recompute=1)
+    r0, _, loss0, _ = check_step(dims, batch, "f32", stddev=0.02)
+    assert r1.h.t5_workspace_bytes() < r0.h.t5_workspace_bytes()
+    assert abs(loss1[0] - loss0[0]) <= 1e-6 * abs(loss0[0])
+    check_step(dims, batch, "bf16", floor=True, recompute=1)
+    dims = WL.model_dims("xl", **LARGE["xl"])
+    check_step(dims, WL.make_batch(dims), "bf16", floor=True, recompute=1)
+    dims = WL.model_dims("declm", **LARGE["declm"])
+    check_step(dims, WL.make_batch(dims), "bf16", floor=True, recompute=1)
 
 
 def test_all_padding_gives_zero():
