@@ -1029,27 +1029,6 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
   }
   if (warp == 8) tmem_alloc(&bars->tmem, kTmemCols);
   const int span = p.Tq + p.Tk - 1;
-  if (warp < 8) {
-    // One batched fill of the four per-CTA tables (contiguous in shared memory), every global load in flight at
-    // once.  Bias: distance of (key j = k0 + row, query q) is j - q, window index w = row - q + tqp in [1, tqp + 127].
-    const int64_t bh = (int64_t)(b * p.H + h) * p.Tq;
-    const int nb = tqp + 128;
-    auto table = [&](int x) -> uint32_t {
-      if (x < nb) {
-        int g = (x - tqp) + k0 + p.Tq - 1;
-        return __float_as_uint((p.bias_delta && g >= 0 && g < span) ? p.bias_delta[(int64_t)h * span + g] * kLog2e : 0.f);
-      }
-      x -= nb;
-      if (x < tqp) return __float_as_uint(x < p.Tq ? p.lse[bh + x] * kLog2e : -INFINITY);
-      x -= tqp;
-      if (x < tqp) return __float_as_uint(x < p.Tq ? p.delta[bh + x] : 0.f);
-      x -= tqp;
-      return (uint32_t)(x < p.Tq ? p.code_q[b * p.Tq + x] : 0);
-    };
-    fill_batched<kKvfSoftmaxThreads, uint32_t, decltype(table), 9>((uint32_t*)bias_s, nb + 3 * tqp, tid, table);
-    if (want_db)
-      for (int w = tid; w < nb; w += kKvfSoftmaxThreads) dbias_s[w] = 0.f;
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -1141,6 +1120,29 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
     const int quad = warp & 3, half = warp >> 2, row = quad * 32 + lane;
     const int j = k0 + row;
     const int ck = j < p.Tk ? p.code_k[b * p.Tk + j] : 0;
+    {
+      // The per-CTA tables are filled here, by the softmax warps alone and behind their own barrier: the loads
+      // and the first S^T / dP^T MMAs of the other two warps run meanwhile.  One batched fill of the four tables
+      // (contiguous in shared memory), every global load in flight at once.  Bias: distance of (key j = k0 + row, query q) is j - q, window index w = row - q + tqp in [1, tqp + 127].
+      const int64_t bh = (int64_t)(b * p.H + h) * p.Tq;
+      const int nb = tqp + 128;
+      auto table = [&](int x) -> uint32_t {
+        if (x < nb) {
+          int g = (x - tqp) + k0 + p.Tq - 1;
+          return __float_as_uint((p.bias_delta && g >= 0 && g < span) ? p.bias_delta[(int64_t)h * span + g] * kLog2e : 0.f);
+        }
+        x -= nb;
+        if (x < tqp) return __float_as_uint(x < p.Tq ? p.lse[bh + x] * kLog2e : -INFINITY);
+        x -= tqp;
+        if (x < tqp) return __float_as_uint(x < p.Tq ? p.delta[bh + x] : 0.f);
+        x -= tqp;
+        return (uint32_t)(x < p.Tq ? p.code_q[b * p.Tq + x] : 0);
+      };
+      fill_batched<kKvfSoftmaxThreads, uint32_t, decltype(table), 9>((uint32_t*)bias_s, nb + 3 * tqp, tid, table);
+      if (want_db)
+        for (int w = tid; w < nb; w += kKvfSoftmaxThreads) dbias_s[w] = 0.f;
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+    }
     const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
     const float sc2 = p.scale * kLog2e;
     const bool has_bias = p.bias_delta != nullptr;
