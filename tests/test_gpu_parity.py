@@ -259,8 +259,6 @@ def test_step_activation_recomputation():
     check_step(dims, batch, "bf16", floor=True, recompute=1)
     dims = WL.model_dims("xl", **LARGE["xl"])
     check_step(dims, WL.make_batch(dims), "bf16", floor=True, recompute=1)
-    dims = WL.model_dims("declm", **LARGE["declm"])
-    check_step(dims, WL.make_batch(dims), "bf16", floor=True, recompute=1)
 
 
 def test_all_padding_gives_zero():
