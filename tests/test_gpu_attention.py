@@ -78,6 +78,9 @@ CASES = [
 @pytest.mark.parametrize("B,H,Tq,Tk,dk,causal,use_bias,mode", CASES + [
     (1, 2, 640, 640, 64, True, True, "packed"),
     (2, 2, 50, 330, 64, False, True, "pad"),
+    # degenerate extents: one query, one key
+    (1, 1, 1, 40, 64, False, True, "full"),
+    (1, 2, 129, 1, 64, False, False, "full"),
     # large scores (scale 1): row maxima move by more than the forward kernel's lazy-rescale threshold between tiles
     (1, 2, 448, 448, 64, False, True, "full_hot"),
 ])
@@ -149,7 +152,10 @@ def test_attention_forward_backward(impl, B, H, Tq, Tk, dk, causal, use_bias, mo
     for name, got, ref, T in (("dq", dq, rdq, Tq), ("dk", dk_t, rdk, Tk), ("dv", dv_t, rdv, Tk)):
         g = f64(got, T)
         assert np.isfinite(g).all(), name
-        assert np.abs(g - ref).max() <= 2e-2 * np.abs(ref).max(), (name, np.abs(g - ref).max(), np.abs(ref).max())
+        # with a single key the softmax is the constant 1 and dS, dq, dk are identically zero in exact arithmetic:
+        # what the kernels leave there is the float32 rounding residue of dP - delta, far below the inputs' scale
+        floor = 1e-4 if Tk == 1 else 0.0
+        assert np.abs(g - ref).max() <= 2e-2 * np.abs(ref).max() + floor, (name, np.abs(g - ref).max(), np.abs(ref).max())
     if use_bias:
         g = dbias.cpu().numpy()
         if far:
