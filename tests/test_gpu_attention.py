@@ -167,3 +167,25 @@ def test_attention_forward_backward(impl, B, H, Tq, Tk, dk, causal, use_bias, mo
                 a[:, c - far] = a[:, :c - far + 1].sum(axis=1)
                 a[:, :c - far] = 0
         assert np.abs(g - rdb).max() <= 2e-2 * np.abs(rdb).max()
+
+
+def test_onepass_backward_rejects_bad_scratch():
+    """The one-pass backward refuses a scratch buffer that is too small or a head width it does not cover,
+    before anything is launched."""
+    B, H, Tq, Tk, dk = 1, 2, 128, 128, 64
+    I = H * dk
+    bf = torch.bfloat16
+    t = torch.zeros(B * Tq, I, dtype=bf, device=DEV)
+    f32 = torch.zeros(B * Tq, I, dtype=torch.float32, device=DEV)
+    lse = torch.zeros(B, H, Tq, dtype=torch.float32, device=DEV)
+    codes = torch.ones(B, Tq, dtype=torch.int32, device=DEV)
+    need = Bd.t5_attention_ds_scratch_bytes(B, H, Tq, Tk)
+    assert need == B * H * 128 * 128 * 2
+    small = torch.zeros(need // 2 - 64, dtype=bf, device=DEV)
+    with pytest.raises(Bd.T5Error):
+        Bd.t5_attention_backward_onepass(B, H, Tq, Tk, dk, False, 1.0, t, t, t, t, f32, lse, codes, codes, None,
+                                         t, t, t, t, lse, None, 0, small)
+    ok = torch.zeros(need // 2, dtype=bf, device=DEV)
+    with pytest.raises(Bd.T5Error):
+        Bd.t5_attention_backward_onepass(B, H, Tq, Tk, 32, False, 1.0, t, t, t, t, f32, lse, codes, codes, None,
+                                         t, t, t, t, lse, None, 0, ok)
