@@ -212,7 +212,10 @@ T5_API int t5_gemm(int32_t dtype, int32_t impl, int32_t M, int32_t N, int32_t K,
  * backward reads for delta = rowsum(dO * O).  Backward writes
  * dq, dk, dv, uses d_delta [B,H,Tq] as scratch and ADDS dS summed along
  * diagonals into d_dbias_delta (may be NULL).  impl 0 = SIMT kernels,
- * 1 = tcgen05 kernels (bfloat16, d_kv 64 or 128). */
+ * 1 = tcgen05 kernels (bfloat16, d_kv 64 or 128).  The tcgen05 forward leaves
+ * out key tiles whose range of position codes does not meet the range of a
+ * CTA's 128 query rows (packed rows); the training step switches that
+ * bookkeeping off for batches without segment ids, this entry point keeps it on. */
 T5_API int t5_attention(int32_t dtype, int32_t impl, int32_t backward, int32_t B, int32_t H, int32_t Tq,
                         int32_t Tk, int32_t d_kv, int32_t causal, float scale, const void* d_q, int32_t ldq,
                         const void* d_k, int32_t ldk, const void* d_v, int32_t ldv, void* d_o, int32_t ldo,

@@ -48,6 +48,7 @@ struct TcParams {
   float scale;
   int* status;
   int bias_far;              // see AttnArgs::bias_far
+  int packed;                // see AttnArgs::packed
 };
 
 
@@ -112,7 +113,7 @@ struct FwdLayout {
   static constexpr int kQ = 0, kK = kQBytes, kV = kK + kKVBytes, kPo = kV + kKVBytes, kMisc = kPo + kP;
   static int bytes(int Tk) {
     int tkp = (Tk + 63) / 64 * 64;
-    return kMisc + (tkp + 128) * 4 + tkp * 4 + (int)sizeof(Bars) + 1024 + 64;
+    return kMisc + (tkp + 128) * 4 + tkp * 4 + (tkp / 64 + 9) * 4 + (int)sizeof(Bars) + 1024 + 64;
   }
 };
 
@@ -126,7 +127,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
   const int tkp = (p.Tk + 63) / 64 * 64;
   float* bias_s = (float*)(smem + L::kMisc);          // [tkp + 128], entry (key - row + 127), log2 units
   int* codes_s = (int*)(bias_s + tkp + 128);          // [tkp]
-  Bars* bars = (Bars*)(((uintptr_t)(codes_s + tkp) + 15) & ~(uintptr_t)15);
+  int* tiles_s = codes_s + tkp;                       // [tkp / 64] key tiles this CTA visits, then 8 + 1 scratch words
+  const int n_tiles_cap = tkp / 64;
+  Bars* bars = (Bars*)(((uintptr_t)(tiles_s + n_tiles_cap + 9) + 15) & ~(uintptr_t)15);
   volatile int* abort_flag = &bars->abort_flag;
 
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -201,20 +204,63 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
 
   const int i = q0 + tid;
   const int cq = i < p.Tq ? p.code_q[b * p.Tq + i] : 0;
+  // Key tiles worth visiting (packed rows only).  A pair (query, key) is valid only if both carry the same non-zero
+  // position code, so a key tile whose range of non-zero codes does not meet the range of this CTA's rows holds no
+  // valid pair (other segments) and is left out.  Tile 0 always stays: its loads and S = Q K^T went out during the
+  // set-up.  Every warp counts the list, warp 0 writes it.
+  int n_act = n_kt;
+  if (p.packed) {
+    int* rng = tiles_s + n_tiles_cap;                  // [8]: (lo, hi) of each warp's rows
+    int lo = cq ? cq : 0x7fffffff, hi = cq;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = ::max(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if ((tid & 31) == 0) { rng[2 * warp] = lo; rng[2 * warp + 1] = hi; }
+    __syncthreads();
+    const int lane = tid & 31;
+    int qlo = 0x7fffffff, qhi = 0;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      qlo = min(qlo, rng[2 * w]);
+      qhi = ::max(qhi, rng[2 * w + 1]);
+    }
+    n_act = 0;
+    for (int base = 0; base < n_kt; base += 2) {       // 16 lanes per tile, one 16-byte load each
+      const int t = base + (lane >> 4);
+      int klo = 0x7fffffff, khi = 0;
+      if (t < n_kt) {
+        const int4 c = *reinterpret_cast<const int4*>(codes_s + t * 64 + (lane & 15) * 4);
+        klo = min(min(c.x ? c.x : 0x7fffffff, c.y ? c.y : 0x7fffffff), min(c.z ? c.z : 0x7fffffff, c.w ? c.w : 0x7fffffff));
+        khi = ::max(::max(c.x, c.y), ::max(c.z, c.w));
+      }
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) {
+        klo = min(klo, __shfl_xor_sync(0xffffffffu, klo, o));
+        khi = ::max(khi, __shfl_xor_sync(0xffffffffu, khi, o));
+      }
+      const bool active = t < n_kt && (t == 0 || (khi > 0 && khi >= qlo && klo <= qhi));
+      const unsigned m = __ballot_sync(0xffffffffu, active) & 0x00010001u;      // one vote per half warp
+      if (warp == 0 && active && (lane & 15) == 0) tiles_s[n_act + ((lane >> 4) & (m & 1u))] = t;
+      n_act += __popc(m);
+    }
+    __syncthreads();                                   // warp 0's list is visible to the thread that issues loads
+  }
   float m_run = -INFINITY, l_run = 0.f;
   const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
   const float sc2 = p.scale * kLog2e;
   const bool has_bias = p.bias_delta != nullptr;
 
-  for (int t = 0; t < n_kt && ok; ++t) {
-    const int k0 = t * 64;
-    ok = mbar_wait(bar_m, ph_m, abort_flag, p.status, 12);      // S(t) ready, PV(t-1) done
+  for (int u = 0; u < n_act && ok; ++u) {
+    const int t = p.packed ? tiles_s[u] : u, k0 = t * 64;
+    ok = mbar_wait(bar_m, ph_m, abort_flag, p.status, 12);      // S of this tile ready, PV of the previous one done
     ph_m ^= 1;
     if (!ok) break;
     tc_fence_after();
     if (tid == 0) {
-      if (t + 1 < n_kt) load_k(t + 1);       // K buffer: S(t) has consumed it
-      if (t > 0) load_v(t);                  // V buffer: PV(t-1) has consumed it
+      if (u + 1 < n_act) load_k(p.packed ? tiles_s[u + 1] : u + 1);   // K buffer: S of this tile has consumed it
+      if (u > 0) load_v(t);                        // V buffer: PV of the previous tile has consumed it
     }
     // ---- softmax of this 64-key tile (scores in log2 units)
     const int tcode = tile_code64(codes_s + k0, tid & 31);
@@ -267,7 +313,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
     const float m_eff = m_new == -INFINITY ? 0.f : m_new;      // a row with no valid key so far: exp2(-inf - 0) = 0
     const float corr = ex2_approx(m_run - m_eff);
     // rescale the accumulator rows of this warp if any of their reference points moved
-    if (t > 0 && warp_moves) {
+    if (u > 0 && warp_moves) {
 #pragma unroll
       for (int c = 0; c < DK / 32; ++c) {
         uint32_t r[32];
@@ -306,8 +352,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
-          umma_bf16_lo(tmem_base + 64, lP + ((ks * 32) >> 4), lV + ((ks * 2048) >> 4), idesc_pv, (t | ks) != 0);
-        if (t + 1 < n_kt) good = issue_s();
+          umma_bf16_lo(tmem_base + 64, lP + ((ks * 32) >> 4), lV + ((ks * 2048) >> 4), idesc_pv, (u | ks) != 0);
+        if (u + 1 < n_act) good = issue_s();
         if (good) umma_commit(bar_m);
       }
     }
@@ -1480,6 +1526,7 @@ TcParams base_params(const AttnArgs& a, int* status) {
   TcParams p{};
   p.lse = a.lse; p.delta = a.delta; p.code_q = a.code_q; p.code_k = a.code_k; p.bias_delta = a.bias_delta;
   p.bias_far = a.bias_far;
+  p.packed = a.packed;
   p.dbias_delta = a.dbias_delta; p.B = a.B; p.H = a.H; p.Tq = a.Tq; p.Tk = a.Tk; p.causal = a.causal;
   p.scale = a.scale; p.status = status;
   return p;

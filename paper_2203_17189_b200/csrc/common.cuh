@@ -107,6 +107,9 @@ struct AttnArgs {
   // one pass over the scores (dK, dV and a bf16 copy of dS^T in this buffer) and takes dQ from the stored dS
   void* ds_scratch = nullptr;
   int64_t ds_bytes = 0;
+  // non-zero: rows may hold several segments (packed examples).  The tcgen05 forward then leaves out key tiles whose
+  // range of position codes does not meet the range of the CTA's query rows; 0 skips that bookkeeping.
+  int packed = 0;
 };
 int64_t attn_tc_ds_scratch_bytes(int B, int H, int Tq, int Tk);
 bool attn_tc_onepass_supported(const AttnArgs& a);   // the backward will take the one-pass route

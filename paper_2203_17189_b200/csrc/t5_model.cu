@@ -274,6 +274,7 @@ struct Ctx {
   const char* where;
   int64_t launches;
   int sk_next;        // next unused flag slice
+  int packed;         // the batch carries segment ids
 };
 
 enum { CAT_GEMM = 0, CAT_ATTN_FWD, CAT_ATTN_BWD, CAT_NORM, CAT_GEGLU, CAT_XENT, CAT_EMBED, CAT_MISC };
@@ -400,6 +401,7 @@ void attn_args(Ctx& cx, const AttnWs& a, const AttnGeom& gm, bool cross, AttnArg
   t.B = cx.B; t.H = c.n_heads; t.Tq = gm.Tq; t.Tk = gm.Tk; t.dk = c.d_kv;
   t.code_q = gm.code_q; t.code_k = gm.code_k; t.causal = gm.causal;
   t.bias_delta = gm.bias; t.scale = c.attn_scale;
+  t.packed = cx.packed;
 }
 
 // x_out = x + Attn(RMS(x))
@@ -708,6 +710,7 @@ int begin_call(t5_handle* h, const void* params, const t5_batch* b, void* ws, in
                 (long long)w->bytes);
   cx->h = h; cx->params = params; cx->grads = nullptr; cx->st = (cudaStream_t)stream; cx->w = w;
   cx->B = b->B; cx->Te = Te; cx->Td = b->Td; cx->err = cudaSuccess; cx->where = ""; cx->launches = 0; cx->sk_next = 0;
+  cx->packed = (b->d_enc_segment_ids != nullptr || b->d_dec_segment_ids != nullptr) ? 1 : 0;
   return T5_OK;
 }
 
@@ -937,6 +940,7 @@ int t5_attention(int32_t dtype, int32_t impl, int32_t backward, int32_t B, int32
   a.B = B; a.H = H; a.Tq = Tq; a.Tk = Tk; a.dk = d_kv; a.code_q = d_code_q; a.code_k = d_code_k; a.causal = causal;
   a.bias_delta = d_bias_delta; a.scale = scale; a.dO = d_do; a.lddo = lddo; a.dQ = d_dq; a.dK = d_dk; a.dV = d_dv;
   a.lddq = lddq; a.lddk = lddk; a.lddv = lddv; a.delta = d_delta; a.dbias_delta = d_dbias_delta;
+  a.packed = 1;      // the codes may describe packed rows: keep the tile-skipping bookkeeping on
   cudaStream_t st = (cudaStream_t)stream;
   cudaError_t e;
   if (impl == 0) {
