@@ -199,12 +199,11 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
       tma_load_3d(smem + L::kK + c * 8192, &mk, h * DK + c * 64, 0, b, bar_k);
     }
     load_v(0);
-    if (issue_s()) umma_commit(bar_m);
   }
 
   const int i = q0 + tid;
   const int cq = i < p.Tq ? p.code_q[b * p.Tq + i] : 0;
-  // Key tiles worth visiting (packed rows only).  A pair (query, key) is valid only if both carry the same non-zero
+  // Key tiles worth visiting (packed rows only; done while the first loads are in flight).  A pair (query, key) is valid only if both carry the same non-zero
   // position code, so a key tile whose range of non-zero codes does not meet the range of this CTA's rows holds no
   // valid pair (other segments) and is left out.  Tile 0 always stays: its loads and S = Q K^T went out during the
   // set-up.  Every warp counts the list, warp 0 writes it.
@@ -247,6 +246,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
     }
     __syncthreads();                                   // warp 0's list is visible to the thread that issues loads
   }
+  if (tid == 0 && issue_s()) umma_commit(bar_m);       // S of tile 0 as soon as Q and K(0) have landed
   float m_run = -INFINITY, l_run = 0.f;
   const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
   const float sc2 = p.scale * kLog2e;
