@@ -10,6 +10,7 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu)")
+    config.addinivalue_line("markers", "slow: a GPU test whose oracle run takes minutes")
 
 
 def _has_cuda():

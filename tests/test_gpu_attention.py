@@ -30,6 +30,36 @@ def make_codes(rng, B, T, mode):
     return c
 
 
+def make_cross_codes(rng, B, Tq, Tk, mode):
+    """Packed rows with different query and key lengths (cross-attention of packed examples): the same
+    examples, in the same order, on both sides, each side with its own lengths.
+    'xpacked': ids 1.. in order;  'xmiss0': the queries hold only the later examples, so the first key tiles
+    contain no key any query row may attend;  'xnonmono': example ids are not increasing along the row."""
+    cq = np.zeros((B, Tq), dtype=np.int32)
+    ck = np.zeros((B, Tk), dtype=np.int32)
+    for b in range(B):
+        n = int(rng.integers(3, 6))
+        ids = np.arange(1, n + 1)
+        if mode == "xnonmono":
+            ids = rng.permutation(ids) + int(rng.integers(0, 3))
+
+        def cut(T, frac_used):
+            edges = np.sort(rng.choice(np.arange(1, int(T * frac_used)), size=n - 1, replace=False))
+            return np.concatenate([[0], edges, [int(T * frac_used)]])
+        ek, eq = cut(Tk, 0.93), cut(Tq, 0.9)
+        for s in range(n):
+            ck[b, ek[s]:ek[s + 1]] = ids[s]
+        if mode == "xmiss0":
+            # queries: only the last two examples, spread over the whole used part of the row
+            half = eq[-1] // 2
+            cq[b, :half] = ids[n - 2]
+            cq[b, half:eq[-1]] = ids[n - 1]
+        else:
+            for s in range(n):
+                cq[b, eq[s]:eq[s + 1]] = ids[s]
+    return cq, ck
+
+
 def reference(q, k, v, do, code_q, code_k, bias_delta, causal, scale, H, dk):
     """Oracle arithmetic per (b, h): masked softmax attention and its gradients (float64)."""
     B, Tq = code_q.shape
@@ -83,6 +113,11 @@ CASES = [
     (1, 2, 129, 1, 64, False, False, "full"),
     # large scores (scale 1): row maxima move by more than the forward kernel's lazy-rescale threshold between tiles
     (1, 2, 448, 448, 64, False, True, "full_hot"),
+    # packed rows with different query / key lengths and several examples on both sides
+    (3, 2, 114, 512, 64, False, False, "xpacked"),
+    (2, 2, 114, 512, 64, False, False, "xmiss0"),
+    (2, 2, 300, 700, 64, False, True, "xnonmono"),
+    (1, 2, 260, 520, 128, False, False, "xmiss0"),
 ])
 def test_attention_forward_backward(impl, B, H, Tq, Tk, dk, causal, use_bias, mode):
     rng = np.random.default_rng(B * 1000 + Tq + Tk + dk)
@@ -102,10 +137,13 @@ def test_attention_forward_backward(impl, B, H, Tq, Tk, dk, causal, use_bias, mo
         kv = rnd(B * Tk, 2 * I, s=0.7)
         k, v = kv[:, :I], kv[:, I:]
     do = rnd(B * Tq, I)
-    code_k = make_codes(rng, B, Tk, mode)
-    code_q = code_k if Tq == Tk else make_codes(rng, B, Tq, "pad" if mode != "full" else "full")
-    if mode == "packed" and Tq != Tk:
-        code_q = np.minimum(code_q, 1)
+    if mode.startswith("x"):
+        code_q, code_k = make_cross_codes(rng, B, Tq, Tk, mode)
+    else:
+        code_k = make_codes(rng, B, Tk, mode)
+        code_q = code_k if Tq == Tk else make_codes(rng, B, Tq, "pad" if mode != "full" else "full")
+        if mode == "packed" and Tq != Tk:
+            code_q = np.minimum(code_q, 1)
     bias = (rng.standard_normal((H, Tq + Tk - 1)) * 0.5).astype(np.float32) if use_bias else None
     scale = 1.0 if hot else (0.25 if dk == 64 else 0.2)
     # one-pass backward with a saturated bias: constant beyond +-far, whose dS mass is then booked at +-far
