@@ -305,10 +305,15 @@ def test_step_xl_full_depth_stated_bars_bf16():
     """The XL model at its real depth (24 + 24 layers, every launch of the schedule, the workspace
     reuse across 48 layers, the encoder-output gradient accumulated over 24 cross-attention blocks) on one batch
     row against the oracle (float32 arithmetic: the float64 parameter and gradient copies of 2.8 G parameters
-    would not fit a modest host), attention logits of order one, stated bars."""
+    would not fit a modest host), attention logits of order one.  Cosine >= 0.999 for every tensor; the error
+    bar is the larger of 2e-2 and twice what the oracle itself loses when its operands are rounded to bfloat16
+    (48 layers deep, on a single row, that loss is 3.5e-2 for a few q / k projections of the last layers)."""
     dims = WL.model_dims("xl", batch=1)
     batch = WL.make_batch(dims)
-    check_step(dims, batch, "bf16", attn_scale=dims["d_kv"] ** -0.5, floor=False, oracle_dtype=np.float32)
+    tab = {}
+    check_step(dims, batch, "bf16", attn_scale=dims["d_kv"] ** -0.5, floor=True, oracle_dtype=np.float32,
+               table_out=tab)
+    assert min(v[0] for v in tab.values()) >= 0.999
 
 
 def test_step_activation_recomputation():
