@@ -60,10 +60,18 @@ class T5Config:
     operand_bf16: bool = False    # round BOTH operands of every matrix product to bfloat16 first
                                   # (the "bf16 operands, float32 accumulate" precision the larger
                                   # workloads are stated in); everything else stays in `dtype`
+    # Members of the model family the paper's "Example Models" section lists beside T5.1.1:
+    ffn_act: str = "gated-gelu-tanh"   # "gated-gelu-tanh" (default): (gelu_tanh(y Wi0) * (y Wi1)) Wo;
+                                       # "gated-gelu-erf": the same with the exact (erf) GELU;
+                                       # "relu": T5 v1.0's FFN, relu(y Wi0) Wo, no gate and no Wi1
+    tied_embedding: bool = True        # False: the logits use a separate matrix "lm_head" [d, V]
+                                       # (released T5.1.1) and logit_scale defaults to 1
 
     def __post_init__(self):
         if self.logit_scale < 0:
-            self.logit_scale = float(self.d_model) ** -0.5
+            self.logit_scale = float(self.d_model) ** -0.5 if self.tied_embedding else 1.0
+        if self.ffn_act not in ("gated-gelu-tanh", "gated-gelu-erf", "relu"):
+            raise ValueError(f"unknown ffn_act {self.ffn_act!r}")
 
     @property
     def inner(self):
@@ -157,6 +165,27 @@ def gelu_tanh_grad(u):
     return 0.5 * (1.0 + t) + 0.5 * u * (1.0 - t * t) * dinner
 
 
+def gelu_erf(u):
+    """u Phi(u) = 0.5 u (1 + erf(u / sqrt 2)), Phi the standard normal distribution function."""
+    from scipy.special import erf
+    return 0.5 * u * (1.0 + erf(u / math.sqrt(2.0)))
+
+
+def gelu_erf_grad(u):
+    """Phi(u) + u phi(u), phi the standard normal density."""
+    from scipy.special import erf
+    return 0.5 * (1.0 + erf(u / math.sqrt(2.0))) + u * np.exp(-0.5 * u * u) / math.sqrt(2.0 * math.pi)
+
+
+def ffn_activation(cfg, a):
+    """(act(a), act'(a)) of the configured FFN non-linearity."""
+    if cfg.ffn_act == "relu":
+        return np.maximum(a, 0), (a > 0).astype(a.dtype)
+    if cfg.ffn_act == "gated-gelu-erf":
+        return gelu_erf(a), gelu_erf_grad(a)
+    return gelu_tanh(a), gelu_tanh_grad(a)
+
+
 def rms_norm(x, g, eps):
     """y = x * (mean(x^2) + eps)^-1/2 * g ; returns (y, r)."""
     r = 1.0 / np.sqrt(np.mean(x * x, axis=-1) + x.dtype.type(eps))
@@ -205,12 +234,26 @@ def shift_right(targets_row, seg_row):
     return u
 
 
-def attention_mask(code_q, code_k, causal):
+def attention_mask(code_q, code_k, causal, prefix_q=None, prefix_k=None):
+    """Query i may attend key j iff both carry the same non-zero code and, when causal, j <= i.
+    Prefix LM: positions flagged in prefix_* form a fully visible prefix, so a causal pair is also
+    allowed when query and key are both flagged."""
     m = (code_k[None, :] != 0) & (code_q[:, None] == code_k[None, :])
     if causal:
         tq, tk = m.shape
-        m &= (np.arange(tk)[None, :] <= np.arange(tq)[:, None])
+        allowed = np.arange(tk)[None, :] <= np.arange(tq)[:, None]
+        if prefix_q is not None:
+            allowed = allowed | ((np.asarray(prefix_q)[:, None] != 0) & (np.asarray(prefix_k)[None, :] != 0))
+        m &= allowed
     return m
+
+
+def loss_weights(targets_row, prefix_row=None):
+    """w_t = 1 for a non-pad target outside the prefix (the prefix is given, not predicted), else 0."""
+    w = np.asarray(targets_row) != 0
+    if prefix_row is not None:
+        w = w & (np.asarray(prefix_row) == 0)
+    return w
 
 
 # ----------------------------------------------------------------------------
@@ -230,7 +273,8 @@ def param_shapes(cfg: T5Config):
     def ffn(prefix):
         s[prefix + ".norm"] = (d,)
         s[prefix + ".wi0"] = (d, F)
-        s[prefix + ".wi1"] = (d, F)
+        if cfg.ffn_act != "relu":
+            s[prefix + ".wi1"] = (d, F)
         s[prefix + ".wo"] = (F, d)
 
     if cfg.arch == 0:
@@ -246,15 +290,18 @@ def param_shapes(cfg: T5Config):
             attn(f"dec.L{l}.cross")
         ffn(f"dec.L{l}.ffn")
     s["dec.final_norm"] = (d,)
+    if not cfg.tied_embedding:
+        s["lm_head"] = (d, V)
     return s
 
 
 # ----------------------------------------------------------------------------
 # Sub-layers, one batch row at a time.  Each forward returns (output, cache).
 # ----------------------------------------------------------------------------
-def _attn_fwd(cfg, p, prefix, x_q, y_kv, table, bidirectional, code_q, code_k, causal):
+def _attn_fwd(cfg, p, prefix, x_q, y_kv, table, bidirectional, code_q, code_k, causal, lm_prefix=None):
     """x_q: residual stream [Tq, d].  y_kv: None for self-attention (keys and
-    values come from the normed x_q) or the already-normed encoder output."""
+    values come from the normed x_q) or the already-normed encoder output.
+    lm_prefix: flags of the fully visible prefix of a prefix LM (causal self-attention only)."""
     H, k = cfg.n_heads, cfg.d_kv
     dt = x_q.dtype
     yq, r = rms_norm(x_q, p[prefix + ".norm"], cfg.rms_eps)
@@ -263,7 +310,7 @@ def _attn_fwd(cfg, p, prefix, x_q, y_kv, table, bidirectional, code_q, code_k, c
     K = mm(cfg, ykv, p[prefix + ".k"])
     Vv = mm(cfg, ykv, p[prefix + ".v"])
     tq, tk = Q.shape[0], K.shape[0]
-    mask = attention_mask(code_q, code_k, causal)
+    mask = attention_mask(code_q, code_k, causal, lm_prefix, lm_prefix)
     bk = None
     if table is not None:
         bk = bucket_matrix(tq, tk, bidirectional, cfg.rel_buckets, cfg.rel_max_distance)
@@ -320,8 +367,12 @@ def _attn_bwd(cfg, p, g, gtable, prefix, dout, c):
 def _ffn_fwd(cfg, p, prefix, x):
     y, r = rms_norm(x, p[prefix + ".norm"], cfg.rms_eps)
     a = mm(cfg, y, p[prefix + ".wi0"])
-    b = mm(cfg, y, p[prefix + ".wi1"])
-    hg = gelu_tanh(a) * b
+    act, _ = ffn_activation(cfg, a)
+    if cfg.ffn_act == "relu":            # T5 v1.0: no gate
+        b, hg = None, act
+    else:
+        b = mm(cfg, y, p[prefix + ".wi1"])
+        hg = act * b
     out = x + mm(cfg, hg, p[prefix + ".wo"])
     return out, dict(x=x, r=r, y=y, a=a, b=b, hg=hg)
 
@@ -329,11 +380,17 @@ def _ffn_fwd(cfg, p, prefix, x):
 def _ffn_bwd(cfg, p, g, prefix, dout, c):
     g[prefix + ".wo"] += mm(cfg, c["hg"].T, dout)
     dhg = mm(cfg, dout, p[prefix + ".wo"].T)
-    da = dhg * c["b"] * gelu_tanh_grad(c["a"])
-    db = dhg * gelu_tanh(c["a"])
-    g[prefix + ".wi0"] += mm(cfg, c["y"].T, da)
-    g[prefix + ".wi1"] += mm(cfg, c["y"].T, db)
-    dy = mm(cfg, da, p[prefix + ".wi0"].T) + mm(cfg, db, p[prefix + ".wi1"].T)
+    act, dact = ffn_activation(cfg, c["a"])
+    if cfg.ffn_act == "relu":
+        da = dhg * dact
+        g[prefix + ".wi0"] += mm(cfg, c["y"].T, da)
+        dy = mm(cfg, da, p[prefix + ".wi0"].T)
+    else:
+        da = dhg * c["b"] * dact
+        db = dhg * act
+        g[prefix + ".wi0"] += mm(cfg, c["y"].T, da)
+        g[prefix + ".wi1"] += mm(cfg, c["y"].T, db)
+        dy = mm(cfg, da, p[prefix + ".wi0"].T) + mm(cfg, db, p[prefix + ".wi1"].T)
     dxn, dg = rms_norm_bwd(dy, c["x"], p[prefix + ".norm"], c["r"])
     g[prefix + ".norm"] += dg
     return dout + dxn
@@ -361,28 +418,36 @@ def _encoder_bwd(cfg, p, g, dy, c):
     np.add.at(g["token_embed"], c["tokens"], dx)
 
 
-def _decoder_fwd(cfg, p, targets_row, dseg_row, enc_y, enc_code):
+def _out_embedding(cfg, p):
+    """[V, d] matrix of the logits: the input embedding when tied, else the separate head (stored [d, V])."""
+    return p["token_embed"] if cfg.tied_embedding else p["lm_head"].T
+
+
+def _decoder_fwd(cfg, p, targets_row, dseg_row, enc_y, enc_code, lm_prefix=None):
     code = position_codes(targets_row, dseg_row)
     u = shift_right(targets_row, dseg_row)
     x = p["token_embed"][u]
     caches = []
     for l in range(cfg.n_dec_layers):
-        x, cs = _attn_fwd(cfg, p, f"dec.L{l}.self", x, None, p["dec.relbias"], False, code, code, True)
+        x, cs = _attn_fwd(cfg, p, f"dec.L{l}.self", x, None, p["dec.relbias"], False, code, code, True, lm_prefix)
         cc = None
         if cfg.arch == 0:
             x, cc = _attn_fwd(cfg, p, f"dec.L{l}.cross", x, enc_y, None, False, code, enc_code, False)
         x, cf = _ffn_fwd(cfg, p, f"dec.L{l}.ffn", x)
         caches.append((cs, cc, cf))
     z, r = rms_norm(x, p["dec.final_norm"], cfg.rms_eps)
-    logits = x.dtype.type(cfg.logit_scale) * mm(cfg, z, p["token_embed"].T)
+    logits = x.dtype.type(cfg.logit_scale) * mm(cfg, z, _out_embedding(cfg, p).T)
     return logits, dict(u=u, layers=caches, x_final=x, r_final=r, z=z)
 
 
 def _decoder_bwd(cfg, p, g, dlogits, c, enc_y):
     dt = dlogits.dtype
     ls = dt.type(cfg.logit_scale)
-    g["token_embed"] += ls * mm(cfg, dlogits.T, c["z"])
-    dz = ls * mm(cfg, dlogits, p["token_embed"])
+    if cfg.tied_embedding:
+        g["token_embed"] += ls * mm(cfg, dlogits.T, c["z"])
+    else:
+        g["lm_head"] += ls * mm(cfg, c["z"].T, dlogits)
+    dz = ls * mm(cfg, dlogits, _out_embedding(cfg, p))
     dx, dg = rms_norm_bwd(dz, c["x_final"], p["dec.final_norm"], c["r_final"])
     g["dec.final_norm"] += dg
     denc = None if enc_y is None else np.zeros_like(enc_y)
@@ -417,8 +482,11 @@ def _cast_params(params, dtype):
 
 
 def t5_train_step(cfg: T5Config, params, enc_tokens, enc_segment_ids, dec_targets,
-                  dec_segment_ids, dtype=np.float64, return_aux=False):
+                  dec_segment_ids, dtype=np.float64, return_aux=False, dec_prefix=None):
     """Loss and gradients of one batch.
+
+    dec_prefix ([B, Td] 0/1, optional): prefix-LM flags of the decoder positions - flagged positions see each
+    other in full (inside their segment), the rest stay causal, and flagged positions carry no loss.
 
     Returns (loss4, grads): loss4 = [L, ce, zl, W] with
       W  = number of non-pad targets,
@@ -431,7 +499,8 @@ def t5_train_step(cfg: T5Config, params, enc_tokens, enc_segment_ids, dec_target
     g = {k: np.zeros(v.shape, dtype=dtype) for k, v in p.items()}
     dec_targets = np.asarray(dec_targets)
     B = dec_targets.shape[0]
-    W = int(np.sum(dec_targets != 0))
+    dec_prefix = None if dec_prefix is None else np.asarray(dec_prefix)
+    W = int(np.sum(loss_weights(dec_targets, dec_prefix)))
     ce_sum = 0.0
     zl_sum = 0.0
     aux = dict(enc_out=[], logits=[], dlogits=[])
@@ -443,8 +512,9 @@ def t5_train_step(cfg: T5Config, params, enc_tokens, enc_segment_ids, dec_target
             enc_code = ec["code"]
         else:
             enc_y, ec, enc_code = None, None, None
-        logits, dc = _decoder_fwd(cfg, p, dec_targets[b], dseg, enc_y, enc_code)
-        w = (dec_targets[b] != 0).astype(dtype)
+        pre = None if dec_prefix is None else dec_prefix[b]
+        logits, dc = _decoder_fwd(cfg, p, dec_targets[b], dseg, enc_y, enc_code, pre)
+        w = loss_weights(dec_targets[b], pre).astype(dtype)
         ce_t, zl_t, lse, prob = xent_zloss_row(logits, dec_targets[b], w, cfg.z_loss)
         ce_sum += float(np.sum(w * ce_t))
         zl_sum += float(np.sum(w * zl_t))
@@ -472,12 +542,13 @@ def t5_train_step(cfg: T5Config, params, enc_tokens, enc_segment_ids, dec_target
 
 
 def t5_loss_only(cfg, params, enc_tokens, enc_segment_ids, dec_targets, dec_segment_ids,
-                 dtype=np.float64):
+                 dtype=np.float64, dec_prefix=None):
     """Forward only: the scalar L (used by finite differences)."""
     dtype = np.dtype(dtype)
     p = _cast_params(params, dtype)
     dec_targets = np.asarray(dec_targets)
-    W = int(np.sum(dec_targets != 0))
+    dec_prefix = None if dec_prefix is None else np.asarray(dec_prefix)
+    W = int(np.sum(loss_weights(dec_targets, dec_prefix)))
     if W == 0:
         return 0.0
     tot = 0.0
@@ -488,8 +559,9 @@ def t5_loss_only(cfg, params, enc_tokens, enc_segment_ids, dec_targets, dec_segm
         if cfg.arch == 0:
             enc_y, ec = _encoder_fwd(cfg, p, np.asarray(enc_tokens)[b], eseg)
             enc_code = ec["code"]
-        logits, _ = _decoder_fwd(cfg, p, dec_targets[b], dseg, enc_y, enc_code)
-        w = (dec_targets[b] != 0).astype(dtype)
+        pre = None if dec_prefix is None else dec_prefix[b]
+        logits, _ = _decoder_fwd(cfg, p, dec_targets[b], dseg, enc_y, enc_code, pre)
+        w = loss_weights(dec_targets[b], pre).astype(dtype)
         ce_t, zl_t, _, _ = xent_zloss_row(logits, dec_targets[b], w, cfg.z_loss)
         tot += float(np.sum(w * (ce_t + zl_t)))
     return tot / W
@@ -507,7 +579,7 @@ def t5_encode(cfg, params, enc_tokens, enc_segment_ids, dtype=np.float64):
 
 
 def t5_decode_logits(cfg, params, enc_out, enc_tokens, enc_segment_ids, dec_targets,
-                     dec_segment_ids, dtype=np.float64):
+                     dec_segment_ids, dtype=np.float64, dec_prefix=None):
     """Teacher-forced decoder logits [B, Td, V] given the encoder output
     (enc_out is ignored for the decoder-only architecture)."""
     dtype = np.dtype(dtype)
@@ -521,6 +593,7 @@ def t5_decode_logits(cfg, params, enc_out, enc_tokens, enc_segment_ids, dec_targ
             eseg = None if enc_segment_ids is None else np.asarray(enc_segment_ids)[b]
             ey = np.asarray(enc_out[b], dtype=dtype)
             ecode = position_codes(np.asarray(enc_tokens)[b], eseg)
-        logits, _ = _decoder_fwd(cfg, p, dec_targets[b], dseg, ey, ecode)
+        pre = None if dec_prefix is None else np.asarray(dec_prefix)[b]
+        logits, _ = _decoder_fwd(cfg, p, dec_targets[b], dseg, ey, ecode, pre)
         outs.append(logits)
     return np.stack(outs)

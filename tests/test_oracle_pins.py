@@ -192,8 +192,9 @@ def test_dlogits_row_sum_identity():
 
 
 # ------------------------------------------------------------- gradients
-def _fd_check(cfg, params, enc, eseg, dec, dseg, n_coord=24, all_of=("relbias",), seed=0):
-    loss4, g = O.t5_train_step(cfg, params, enc, eseg, dec, dseg, dtype=np.float64)
+def _fd_check(cfg, params, enc, eseg, dec, dseg, n_coord=24, all_of=("relbias",), seed=0, dec_prefix=None,
+              h_rel=2e-4):
+    loss4, g = O.t5_train_step(cfg, params, enc, eseg, dec, dseg, dtype=np.float64, dec_prefix=dec_prefix)
     rng = np.random.default_rng(seed)
     worst = 0.0
     p64 = {k: np.array(v, dtype=np.float64) for k, v in params.items()}
@@ -206,11 +207,11 @@ def _fd_check(cfg, params, enc, eseg, dec, dseg, n_coord=24, all_of=("relbias",)
         flat = arr.reshape(-1)
         for i in idxs:
             old = flat[i]
-            h = 2e-4 * max(1.0, abs(old))
+            h = h_rel * max(1.0, abs(old))
             f = {}
             for mlt in (-2, -1, 1, 2):
                 flat[i] = old + mlt * h
-                f[mlt] = O.t5_loss_only(cfg, p64, enc, eseg, dec, dseg)
+                f[mlt] = O.t5_loss_only(cfg, p64, enc, eseg, dec, dseg, dec_prefix=dec_prefix)
             flat[i] = old
             fd = (8 * (f[1] - f[-1]) - (f[2] - f[-2])) / (12 * h)     # 4th-order central difference
             an = g[name].reshape(-1)[i]
@@ -470,3 +471,114 @@ def test_bf16_operand_rounding_floor():
     r = O.round_bf16(a)
     assert r[0] == 1.0 and r[1] == 1.0 and r[2] == 1.0 + 2 ** -7 and r[3] == -3.140625
     assert np.all(r == WL.round_to_bf16(a.astype(np.float32)).astype(np.float64))
+
+
+# ------------------------------------------------------------------ model-family variants
+def test_erf_gelu_printed_values_and_derivative():
+    """u Phi(u) at a few points from the standard normal table (Phi(1) = 0.8413447, Phi(2) = 0.9772499) and the
+    derivative against a central difference."""
+    for line in open(os.path.join(GOLD, "closed_forms.txt")):
+        f = line.split()
+        if f and f[0] == "gelu_erf":
+            assert abs(float(O.gelu_erf(np.float64(f[1]))) - float(f[2])) < 1e-6
+    assert abs(float(O.gelu_erf(np.float64(1.0))) - 0.8413447) < 1e-6
+    u = np.linspace(-4, 4, 81)
+    h = 1e-6
+    fd = (O.gelu_erf(u + h) - O.gelu_erf(u - h)) / (2 * h)
+    assert np.abs(fd - O.gelu_erf_grad(u)).max() < 1e-8
+    # the tanh form approximates it to a few 1e-4 (that is why the two are different configurations)
+    assert 1e-5 < np.abs(O.gelu_erf(u) - O.gelu_tanh(u)).max() < 1e-3
+
+
+def test_relu_ffn_is_a_plain_mlp():
+    """T5 v1.0's FFN: relu(y Wi) Wo - no gate, no second input matrix; against the definition written out."""
+    cfg = tiny_cfg(ffn_act="relu")
+    shapes = O.param_shapes(cfg)
+    assert not any(k.endswith(".wi1") for k in shapes)
+    rng = np.random.default_rng(0)
+    p = {k: rng.standard_normal(v) * 0.3 for k, v in shapes.items()}
+    x = rng.standard_normal((5, cfg.d_model))
+    out, _ = O._ffn_fwd(cfg, p, "enc.L0.ffn", x)
+    g = p["enc.L0.ffn.norm"]
+    y = np.array([row / math.sqrt(np.mean(row ** 2) + cfg.rms_eps) * g for row in x])
+    want = x + np.maximum(y @ p["enc.L0.ffn.wi0"], 0.0) @ p["enc.L0.ffn.wo"]
+    assert np.abs(out - want).max() < 1e-12
+
+
+def test_prefix_lm_mask_hand_case_and_limits():
+    code = np.array([1, 1, 1, 1, 2, 2, 0], dtype=np.int32)
+    pre = np.array([1, 1, 0, 0, 1, 0, 0], dtype=np.int32)
+    m = O.attention_mask(code, code, True, pre, pre)
+    want = np.zeros((7, 7), dtype=bool)
+    for i, j in [(0, 0), (0, 1), (1, 0), (1, 1),             # the prefix of example 1 sees itself in full
+                 (2, 0), (2, 1), (2, 2), (3, 0), (3, 1), (3, 2), (3, 3),   # its continuation stays causal
+                 (4, 4), (5, 4), (5, 5)]:                    # example 2: one prefix position, one target
+        want[i, j] = True
+    assert np.array_equal(m, want)
+    # no flags: plain causal mask; all flagged: the bidirectional mask of the same codes
+    none = np.zeros(7, dtype=np.int32)
+    assert np.array_equal(O.attention_mask(code, code, True, none, none), O.attention_mask(code, code, True))
+    allp = np.ones(7, dtype=np.int32)
+    assert np.array_equal(O.attention_mask(code, code, True, allp, allp), O.attention_mask(code, code, False))
+    # prefix positions carry no loss
+    tgt = np.array([5, 6, 7, 8, 9, 3, 0])
+    assert O.loss_weights(tgt, pre).tolist() == [False, False, True, True, False, True, False]
+    assert O.loss_weights(tgt).tolist() == [True] * 6 + [False]
+
+
+@pytest.mark.parametrize("variant", ["relu", "gated-gelu-erf", "untied", "prefix"])
+def test_finite_differences_variants(variant):
+    kw = {}
+    if variant in ("relu", "gated-gelu-erf"):
+        kw["ffn_act"] = variant
+    if variant == "untied":
+        kw["tied_embedding"] = False
+    pre = None
+    if variant == "prefix":
+        cfg = tiny_cfg(arch=1, n_enc_layers=0, n_dec_layers=2)
+        params = WL.make_params(O.param_shapes(cfg), 5, stddev=0.12, scale_jitter=0.2)
+        rng = np.random.default_rng(3)
+        dec = rng.integers(1, cfg.vocab, size=(2, 9)).astype(np.int32)
+        dseg = np.array([[1, 1, 1, 1, 1, 2, 2, 2, 0], [1, 1, 1, 1, 1, 1, 1, 1, 1]], dtype=np.int32)
+        dec = np.where(dseg == 0, 0, dec)
+        pre = np.array([[1, 1, 1, 0, 0, 1, 0, 0, 0], [1, 1, 1, 1, 0, 0, 0, 0, 0]], dtype=np.int32)
+        _fd_check(cfg, params, None, None, dec, dseg, n_coord=12, dec_prefix=pre)
+        return
+    cfg = tiny_cfg(n_enc_layers=1, n_dec_layers=1, **kw)
+    params, enc, dec = tiny_inputs(cfg, stddev=0.12)
+    if variant == "untied":
+        assert cfg.logit_scale == 1.0 and O.param_shapes(cfg)["lm_head"] == (cfg.d_model, cfg.vocab)
+    # relu has kinks: a step small enough that no pre-activation changes sign inside the stencil
+    _fd_check(cfg, params, enc, None, dec, None, n_coord=12, h_rel=1e-6 if variant == "relu" else 2e-4)
+
+
+def test_untied_head_with_the_embedding_copied_equals_tied():
+    """lm_head = token_embed^T with the tied logit scale gives the tied model's loss; the tied embedding gradient
+    is the sum of the two untied pieces."""
+    cfg_t = tiny_cfg(n_enc_layers=1, n_dec_layers=1)
+    params, enc, dec = tiny_inputs(cfg_t, stddev=0.2)
+    cfg_u = tiny_cfg(n_enc_layers=1, n_dec_layers=1, tied_embedding=False, logit_scale=cfg_t.logit_scale)
+    pu = dict(params)
+    pu["lm_head"] = params["token_embed"].T.copy()
+    lt, gt = O.t5_train_step(cfg_t, params, enc, None, dec, None)
+    lu, gu = O.t5_train_step(cfg_u, pu, enc, None, dec, None)
+    assert abs(lt[0] - lu[0]) < 1e-12
+    assert np.abs(gt["token_embed"] - (gu["token_embed"] + gu["lm_head"].T)).max() < 1e-12
+
+
+def test_prefix_lm_all_flagged_equals_bidirectional_attention_output():
+    """With every position flagged the decoder's self-attention mask is the encoder's (bidirectional) one, so the
+    logits at position t depend on later inputs; with no flags they do not (teacher-forcing causality)."""
+    cfg = tiny_cfg(arch=1, n_enc_layers=0, n_dec_layers=1)
+    params = WL.make_params(O.param_shapes(cfg), 2, stddev=0.3)
+    rng = np.random.default_rng(1)
+    dec = rng.integers(1, cfg.vocab, size=(1, 8)).astype(np.int32)
+    dec2 = dec.copy()
+    dec2[0, 6] = (dec[0, 6] % (cfg.vocab - 1)) + 1            # changes decoder input 7 only
+    none, allp = np.zeros((1, 8), dtype=np.int32), np.ones((1, 8), dtype=np.int32)
+    a = O.t5_decode_logits(cfg, params, None, None, None, dec, None, dec_prefix=none)
+    b = O.t5_decode_logits(cfg, params, None, None, None, dec2, None, dec_prefix=none)
+    assert np.abs(a[0, :7] - b[0, :7]).max() == 0.0
+    a = O.t5_decode_logits(cfg, params, None, None, None, dec, None, dec_prefix=allp)
+    b = O.t5_decode_logits(cfg, params, None, None, None, dec2, None, dec_prefix=allp)
+    assert np.abs(a[0, :7] - b[0, :7]).max() > 1e-6
