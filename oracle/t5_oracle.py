@@ -597,3 +597,21 @@ def t5_decode_logits(cfg, params, enc_out, enc_tokens, enc_segment_ids, dec_targ
         logits, _ = _decoder_fwd(cfg, p, dec_targets[b], dseg, ey, ecode, pre)
         outs.append(logits)
     return np.stack(outs)
+
+
+# ----------------------------------------------------------------------------
+# Optimizer step (the training loop of the paper's "Overall structure" section continues past the gradients;
+# the paper prints no update rule - this is the public AdamW definition with decoupled weight decay).
+# ----------------------------------------------------------------------------
+def adamw_update(theta, m, v, g, step, lr, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0, grad_scale=1.0):
+    """One AdamW step on arrays of equal shape; returns (theta, m, v) after it.
+      g' = grad_scale g;  m = b1 m + (1 - b1) g';  v = b2 v + (1 - b2) g'^2;
+      theta = theta - lr ( (m / (1 - b1^t)) / (sqrt(v / (1 - b2^t)) + eps) + weight_decay theta ),  t = step >= 1."""
+    theta, m, v, g = (np.asarray(a, dtype=np.float64) for a in (theta, m, v, g))
+    g = grad_scale * g
+    m = beta1 * m + (1.0 - beta1) * g
+    v = beta2 * v + (1.0 - beta2) * g * g
+    mhat = m / (1.0 - beta1 ** step)
+    vhat = v / (1.0 - beta2 ** step)
+    theta = theta - lr * (mhat / (np.sqrt(vhat) + eps) + weight_decay * theta)
+    return theta, m, v

@@ -99,7 +99,7 @@ def test_bucket_structure():
 # ------------------------------------------------------- elementwise pieces
 def test_gelu_printed_values_and_derivative():
     for line in open(os.path.join(GOLD, "closed_forms.txt")):
-        if line.startswith("gelu"):
+        if line.startswith("gelu "):
             _, u, v = line.split()
             assert abs(float(O.gelu_tanh(np.float64(u))) - float(v)) < 1e-6
     u = np.linspace(-4, 4, 41)
@@ -582,3 +582,23 @@ def test_prefix_lm_all_flagged_equals_bidirectional_attention_output():
     a = O.t5_decode_logits(cfg, params, None, None, None, dec, None, dec_prefix=allp)
     b = O.t5_decode_logits(cfg, params, None, None, None, dec2, None, dec_prefix=allp)
     assert np.abs(a[0, :7] - b[0, :7]).max() > 1e-6
+
+
+# ------------------------------------------------------------------ optimizer step
+def test_adamw_first_step_closed_form_and_quadratic_descent():
+    """From zero moments the bias-corrected first step is lr (g / (|g| + eps) + wd theta) whatever the betas; on
+    f(theta) = |theta - c|^2 / 2 the iterates approach c; weight decay alone shrinks theta geometrically."""
+    rng = np.random.default_rng(0)
+    th, g = rng.standard_normal(50), rng.standard_normal(50)
+    t1, m1, v1 = O.adamw_update(th, np.zeros(50), np.zeros(50), g, 1, 1e-2, 0.8, 0.95, 1e-8, 0.1)
+    assert np.abs(t1 - (th - 1e-2 * (g / (np.abs(g) + 1e-8) + 0.1 * th))).max() < 1e-12
+    assert np.allclose(m1, 0.2 * g) and np.allclose(v1, 0.05 * g * g)
+    c = rng.standard_normal(8)
+    th, m, v = np.zeros(8), np.zeros(8), np.zeros(8)
+    for t in range(1, 2001):
+        th, m, v = O.adamw_update(th, m, v, th - c, t, 5e-3)
+    assert np.abs(th - c).max() < 2e-2
+    th = np.ones(4)
+    for t in range(1, 11):
+        th, _, _ = O.adamw_update(th, np.zeros(4), np.zeros(4), np.zeros(4), t, 0.1, weight_decay=0.5)
+    assert np.allclose(th, 0.95 ** 10)
