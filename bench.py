@@ -55,6 +55,139 @@ def step_flops(c, B=None):
     return 3.0 * fwd
 
 
+def attention_flops(c, B=None):
+    """The attention share of step_flops: the QK^T and PV contractions, forward + backward (2x forward)."""
+    B = c["batch"] if B is None else B
+    H, k, Te, Td = c["n_heads"], c["d_kv"], c["enc_len"], c["dec_len"]
+    if c["arch"] == 0:
+        fwd = c["n_enc_layers"] * 4 * B * H * Te * Te * k + c["n_dec_layers"] * (2 * B * H * Td * Td * k
+                                                                                     + 4 * B * H * Td * Te * k)
+    else:
+        fwd = c["n_dec_layers"] * 2 * B * H * Td * Td * k
+    return 3.0 * fwd
+
+
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM launches of one XL step, from the ncu
+# capture summarised in profiles/gemm_family_dram_traffic_xl_width.md: a 1+1-layer step was captured (the full
+# step holds 46 GB and 795 GEMM launches), its launches grouped into encoder-layer, decoder-layer and logits GEMMs,
+# and the groups scaled by the layer counts (every layer launches the same shapes).  Valid only for the kernel
+# source the capture ran: keyed by the SHA-1 of csrc/gemm_tcgen05.cu, anything else reports null.
+GEMM_DRAM_TRAFFIC = {
+    # "sha1 of gemm_tcgen05.cu": {"xl": bytes per launch averaged over the 795 GEMM launches of a step}
+    "82862f59288c107006ce738ef2df8b26ace9b209": {"xl": 289.9e6},
+}
+
+
+def gemm_traffic_per_launch(workload):
+    import hashlib
+    src = os.path.join(ROOT, "paper_2203_17189_b200", "csrc", "gemm_tcgen05.cu")
+    try:
+        with open(src, "rb") as f:
+            key = hashlib.sha1(f.read()).hexdigest()
+    except OSError:
+        return None
+    return GEMM_DRAM_TRAFFIC.get(key, {}).get(workload)
+
+
+def write_launch_table(path, records, steps, title):
+    """Per distinct (kernel call, shape): launches per step, time per step, share, and the GEMMs' TFLOP/s."""
+    agg = {}
+    for what, fam, M, N, K, ms in records:
+        a = agg.setdefault((what, M, N, K), [0, 0.0, fam])
+        a[0] += 1
+        a[1] += ms
+    total = sum(a[1] for a in agg.values())
+    with open(path, "w") as f:
+        f.write(f"# {title}\n\n| call | M | N | K | launches/step | ms/step | share | avg us | TFLOP/s |\n|---|---|---|---|---|---|---|---|---|\n")
+        for (what, M, N, K), (n, ms, fam) in sorted(agg.items(), key=lambda kv: -kv[1][1]):
+            tf = f"{2.0 * M * N * K * n / (ms * 1e-3) / 1e12:.0f}" if M and ms > 0 else "-"
+            f.write(f"| {what} | {M or '-'} | {N or '-'} | {K or '-'} | {n / steps:g} | {ms / steps:.3f} | "
+                    f"{ms / total:.3f} | {1e3 * ms / n:.1f} | {tf} |\n")
+        f.write(f"\ntotal {total / steps:.2f} ms per step (sum of per-launch CUDA-event times, {steps} step(s))\n")
+
+
+# ---- the attention entry points on their own (--attention-cases): forward, the backward as two kernels that each
+# recompute the scores (t5_attention, backward = 1) and the one-pass backward (t5_attention_backward_onepass), on the
+# shapes of the XL workload's encoder, cross- and decoder self-attention and of the decoder-only workload
+ATTN_CASES = {
+    # B, H, Tq, Tk, d_kv, causal, bias
+    "enc": (32, 32, 512, 512, 64, False, True),
+    "cross": (32, 32, 114, 512, 64, False, False),
+    "self": (32, 32, 114, 114, 64, True, True),
+    "declm": (8, 16, 2048, 2048, 128, True, True),
+}
+
+
+def attn_time_us(torch, fn, reps):
+    for _ in range(2):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps * 1e3
+
+
+def run_attention_case(name, reps):
+    import torch
+    from paper_2203_17189_b200 import binding as Bd
+    DEV = "cuda:0"
+    B, H, Tq, Tk, dk, causal, use_bias = ATTN_CASES[name]
+    I, bf = H * dk, torch.bfloat16
+    g = torch.Generator(device=DEV)
+    g.manual_seed(1)
+
+    def rnd(*shape, s=1.0):
+        return (torch.randn(*shape, device=DEV, generator=g) * s).to(bf)
+    if Tq == Tk:      # q, k, v as column blocks of one projection output, like the model's layout
+        qkv, dqkv = rnd(B * Tq, 3 * I, s=0.7), torch.empty(B * Tq, 3 * I, dtype=bf, device=DEV)
+        q, k, v = qkv[:, :I], qkv[:, I:2 * I], qkv[:, 2 * I:]
+        dq, dk_, dv = dqkv[:, :I], dqkv[:, I:2 * I], dqkv[:, 2 * I:]
+    else:
+        q, kv = rnd(B * Tq, I, s=0.7), rnd(B * Tk, 2 * I, s=0.7)
+        k, v = kv[:, :I], kv[:, I:]
+        dq, dkv = torch.empty_like(q), torch.empty_like(kv)
+        dk_, dv = dkv[:, :I], dkv[:, I:]
+    do = rnd(B * Tq, I)
+    cq = torch.ones(B, Tq, dtype=torch.int32, device=DEV)
+    ck = torch.ones(B, Tk, dtype=torch.int32, device=DEV)
+    bias, far = None, 0
+    if use_bias:      # constant beyond +-91, like a bias expanded from 32 buckets with maximum distance 128
+        bias = torch.randn(H, Tq + Tk - 1, device=DEV, generator=g) * 0.5
+        c = Tq - 1
+        if c - 91 > 0:
+            far = 91
+            bias[:, c + far:] = bias[:, c + far:c + far + 1]
+            bias[:, :c - far] = bias[:, c - far:c - far + 1]
+    o = torch.empty(B * Tq, I, dtype=bf, device=DEV)
+    o32 = torch.empty(B * Tq, I, dtype=torch.float32, device=DEV)
+    lse = torch.empty(B, H, Tq, dtype=torch.float32, device=DEV)
+    delta = torch.empty_like(lse)
+    dbias = torch.zeros(H, Tq + Tk - 1, dtype=torch.float32, device=DEV) if use_bias else None
+    scratch = torch.empty(Bd.t5_attention_ds_scratch_bytes(B, H, Tq, Tk) // 2, dtype=bf, device=DEV)
+    scale = 0.125
+
+    def fwd():
+        Bd.t5_attention(1, False, B, H, Tq, Tk, dk, causal, scale, q, k, v, o, lse, cq, ck, bias, o32=o32)
+
+    def two():
+        Bd.t5_attention(1, True, B, H, Tq, Tk, dk, causal, scale, q, k, v, o, lse, cq, ck, bias, do=do, dq=dq, dk=dk_,
+                        dv=dv, delta=delta, dbias_delta=dbias, o32=o32)
+
+    def one():
+        Bd.t5_attention_backward_onepass(B, H, Tq, Tk, dk, causal, scale, q, k, v, o, o32, lse, cq, ck, bias, do, dq,
+                                         dk_, dv, delta, dbias, far, scratch)
+    fwd()
+    t_f, t_2, t_1 = attn_time_us(torch, fwd, reps), attn_time_us(torch, two, reps), attn_time_us(torch, one, reps)
+    flops = 4.0 * B * H * Tq * Tk * dk * (0.5 if causal else 1.0)
+    print(f"{name:6s} B{B} H{H} {Tq}x{Tk} d_kv {dk} causal {int(causal)} bias {int(use_bias)}: "
+          f"forward {t_f:.0f} us ({flops / t_f / 1e6:.0f} TFLOP/s), backward two-kernel {t_2:.0f} us, one-pass {t_1:.0f} us")
+
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -207,6 +340,10 @@ def main():
     ap.add_argument("--flags", type=int, default=0)
     ap.add_argument("--recompute", type=int, default=0, choices=[0, 1],
                     help="activation policy (0 keeps everything; the reported number uses 0)")
+    ap.add_argument("--attention-cases", default=None, metavar="enc,cross,self,declm",
+                    help="instead of the step, time the attention calls of the C ABI on these shapes and print a table")
+    ap.add_argument("--launch-table", default=None, metavar="PATH",
+                    help="also write a per-call, per-shape table of the profiled steps' device times (markdown)")
     args = ap.parse_args()
     cfg = WL.model_dims(args.workload)
     if args.batch:
@@ -217,6 +354,13 @@ def main():
         cfg["n_dec_layers"] = args.dec_layers
     if args.impl == "reference":
         run_reference(args, cfg)
+        return
+    if args.attention_cases:
+        import torch
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+        for name in args.attention_cases.split(","):
+            run_attention_case(name, max(args.steps, 1))
         return
 
     import torch
@@ -307,6 +451,10 @@ def main():
     for _ in range(prof_steps):
         step()
     torch.cuda.synchronize()
+    if args.launch_table and rank == 0:
+        write_launch_table(args.launch_table, h.t5_profile_launches(), prof_steps,
+                           f"per-launch CUDA-event times, workload {args.workload}, layers "
+                           f"{cfg['n_enc_layers']}+{cfg['n_dec_layers']}, batch {B}")
     prof = h.t5_profile_read()
     h.t5_profile_enable(False)
     gemm_ms, gemm_flops, gemm_launches = prof["gemm"]
@@ -318,6 +466,9 @@ def main():
     if cfg["dtype"] != "bf16":
         peak_tf = peak_tf / 16.0     # float32 SIMT validation path: not a tensor-core contraction
     achieved_tf = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+    attn_ms = prof["attn_fwd"][0] + prof["attn_bwd"][0]
+    attn_launches = prof["attn_fwd"][2] + prof["attn_bwd"][2]
+    attn_tf = attention_flops(cfg) * prof_steps / (attn_ms * 1e-3) / 1e12 if attn_ms > 0 else 0.0
 
     sec = ms * 1e-3 / args.steps
     value = whole_job_value(tokens_per_step, world, ms, args.steps)
@@ -340,12 +491,24 @@ def main():
                 "d2h_bytes_per_step": 16},
         "gpu_launches": launches * args.steps,
         "clocks": clocks,
-        "roofline": {"kernel": "gemm_tc_kernel (tcgen05)", "bound": "tensor", "achieved": achieved_tf,
+        "roofline": {"kernel": "gemm_tc2_kernel (tcgen05.mma.cta_group::2, CTA pairs; the few shapes it does not "
+                               "take run gemm_tc_kernel)" if cfg["dtype"] == "bf16" else "gemm_simt_kernel",
+                     "bound": "tensor", "achieved": achieved_tf,
                      "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf if peak_tf else None,
-                     "peak_kind": f"{peak_kind} sustained bf16 matmul", "traffic": None,
+                     "peak_kind": f"{peak_kind} sustained bf16 matmul",
+                     "traffic": gemm_traffic_per_launch(args.workload),
+                     "traffic_unit": "DRAM bytes per launch (ncu, 1+1-layer capture scaled by layer counts)",
+                     "algorithmic_per_launch": gemm_flops / max(gemm_launches, 1),
                      "launches_per_step": gemm_launches / prof_steps,
                      "avg_launch_ms": gemm_ms / max(gemm_launches, 1),
                      "share_of_step": gemm_ms / total_prof_ms if total_prof_ms else None},
+        # the attention family (forward, delta, dK/dV/dS, dQ kernels): QK^T and PV FLOPs as in step_flops
+        "roofline_attention": {"kernel": "attn_fwd_tc / attn_bwd_kvf_tc / attn_bwd_dq_ds_tc / attn_delta_tc",
+                               "bound": "tensor", "achieved": attn_tf, "peak": peak_tf, "unit": "TFLOP/s",
+                               "frac": attn_tf / peak_tf if peak_tf else None,
+                               "peak_kind": f"{peak_kind} sustained bf16 matmul", "traffic": None,
+                               "launches_per_step": attn_launches / prof_steps,
+                               "share_of_step": attn_ms / total_prof_ms if total_prof_ms else None},
         "kernel_ms_per_step": {k: v[0] / prof_steps for k, v in prof.items()},
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

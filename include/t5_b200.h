@@ -17,9 +17,13 @@
  *    handle (or for a failed t5_create when passed NULL).
  *  - Pointers named d_* are DEVICE pointers owned by the caller; they must be
  *    16-byte aligned.  Everything else is a host pointer.
- *  - The library allocates no device memory.  All work is enqueued on the
- *    caller's stream (a cudaStream_t passed as void*); no call synchronises
- *    the device.
+ *  - The library allocates no device memory.  All work is ordered by the
+ *    caller's stream (a cudaStream_t passed as void*): kernels are enqueued
+ *    on it, except that the training step runs its weight-gradient GEMMs on
+ *    a second stream owned by the handle, forked from the caller's stream
+ *    and joined back into it before the call returns, so anything enqueued
+ *    on the caller's stream afterwards sees the finished step.  No call
+ *    synchronises the device.
  *  - Token id 0 is padding.  Segment ids are optional (NULL = one example per
  *    row); segment id 0 marks padding in packed rows.  A position's "code" is
  *    0 when its token is padding, else its segment id (1 if unpacked).  Query
@@ -36,7 +40,7 @@
 extern "C" {
 #endif
 
-#define T5_ABI_VERSION 1
+#define T5_ABI_VERSION 2
 
 #if defined(__GNUC__)
 #define T5_API __attribute__((visibility("default")))
@@ -67,22 +71,26 @@ typedef struct {
   float z_loss, rms_eps, attn_scale, logit_scale; /* 1e-4, 1e-6, 1.0, d_model^-1/2 */
   int32_t dtype;            /* 0: float32 everywhere (validation mode);
                                1: bfloat16 parameters/operands, float32 accumulation */
-  int32_t recompute;        /* activation policy: 0 keep everything; 1 do not keep the normed
-                               activations and the gated-GELU product of each sub-layer but
-                               recompute them (one RMSNorm pass, one gated-GELU pass) in the
-                               backward pass right before the weight-gradient GEMMs that read
-                               them: a smaller workspace for a few per cent of step time */
+  int32_t recompute;        /* activation policy: 0 keep everything; 1 do not keep the scaled
+                               operand copy of the residual rows and the gated-GELU product of
+                               each sub-layer but recompute them (one scaling pass, one
+                               gated-GELU pass) in the backward pass right before the
+                               weight-gradient GEMMs that read them: a smaller workspace for a
+                               few per cent of step time */
   int32_t flags;            /* debugging aids for bfloat16 mode: bit 0 = use the plain SIMT
                                GEMM kernel, bit 1 = use the plain SIMT attention kernels,
                                bit 2 = do NOT run the GEMMs on CTA pairs (cta_group::2),
                                bit 3 = keep the gated GELU in separate kernels instead of the GEMM epilogues.
+                               bit 4 = keep the weight-gradient GEMMs on the caller's stream (no second stream).
                                bit 17 = attention backward as two kernels that each recompute the scores
-                               (no dS scratch in the workspace) instead of the one-pass pair.
-                               In float32 mode bits 4..16 round one family of intermediates
-                               to bfloat16 in place (normed activations, projections, context,
-                               FFN pre-activations, gated product, logits, dlogits, residual
-                               gradient copy, dgrad outputs, dcontext, dq/dk/dv, d(gated),
-                               d(pre-activations)) to attribute bfloat16 error */
+                               (no dS scratch in the workspace) instead of the one-pass pair. */
+  /* Members of the model family the paper's "Example Models" section lists beside T5.1.1: */
+  int32_t ffn_act;          /* 0: gated GELU, tanh form (T5.1.1; FFN(y) = (gelu(y Wi0) * (y Wi1)) Wo);
+                               1: ReLU without a gate (T5 v1.0; FFN(y) = relu(y Wi0) Wo, no wi1 tensor);
+                               2: gated GELU, exact (erf) form */
+  int32_t untied_head;      /* 0: the logits use the token embedding (logit_scale d_model^-1/2 by convention);
+                               1: they use a separate tensor lm_head [vocab, embed] (released T5.1.1;
+                               logit_scale 1 by convention) */
 } t5_config;
 
 /* One batch.  All pointers are device pointers to int32 arrays. */
@@ -93,6 +101,9 @@ typedef struct {
   const int32_t* d_dec_targets;      /* [B,Td]; decoder inputs = targets shifted right
                                         (0 at a row or segment start) */
   const int32_t* d_dec_segment_ids;  /* [B,Td] or NULL */
+  const int32_t* d_dec_prefix;       /* [B,Td] 0/1 or NULL.  Prefix LM (the decoder-only model with an
+                                        "inputs" part): flagged positions of a segment see each other in
+                                        full, the rest stay causal, and flagged positions carry no loss */
 } t5_batch;
 
 typedef struct t5_handle t5_handle;
@@ -110,7 +121,8 @@ T5_API const char* t5_last_error(const t5_handle* h);
  *   *.norm / *.final_norm [embed];
  *   enc.L<i>.attn.{q,k,v} [heads*kv, embed]; .o [embed, heads*kv];
  *   *.ffn.{wi0,wi1} [mlp, embed]; .wo [embed, mlp];
- *   dec.L<i>.{self,cross}.* likewise.
+ *   dec.L<i>.{self,cross}.* likewise; lm_head [vocab, embed] last when untied_head = 1;
+ *   no *.ffn.wi1 when ffn_act = 1.
  * Dense weights are stored [out_features, in_features], row-major: a
  * projection computes y[t, o] = sum_i x[t, i] * W[o, i]. */
 T5_API int t5_param_count(const t5_handle* h, int64_t* n_elements);
@@ -143,6 +155,17 @@ T5_API int t5_train_step_fwd_bwd(t5_handle* h, const void* d_params, const t5_ba
                           float* d_grads, float* d_loss4, void* d_workspace,
                           int64_t workspace_bytes, void* stream);
 
+/* The optimizer step that follows the gradients in the paper's training loop ("Overall structure" section; the paper
+ * prints no update rule - this is AdamW with decoupled weight decay).  All buffers are flat, in the parameter layout:
+ * d_master (float32 master weights), d_m, d_v (float32 moments, zero before the first step), d_grads (float32, as
+ * written by t5_train_step_fwd_bwd); d_params receives the master weights rounded to the configured dtype.
+ *   g = grad_scale * grad;  m = beta1 m + (1 - beta1) g;  v = beta2 v + (1 - beta2) g^2;
+ *   master -= lr ( (m / (1 - beta1^step)) / (sqrt(v / (1 - beta2^step)) + eps) + weight_decay master ),  step >= 1.
+ * Weight decay applies to matrices, embeddings and bias tables, not to the 1-D norm scales. */
+T5_API int t5_adamw_update(t5_handle* h, void* d_params, float* d_master, float* d_m, float* d_v,
+                           const float* d_grads, int64_t step, float lr, float beta1, float beta2, float eps,
+                           float weight_decay, float grad_scale, void* stream);
+
 /* Inference method, encoder half: d_enc_out [B,Te,d_model] in the configured
  * dtype = the encoder stack's output after its final norm. */
 T5_API int t5_encode(t5_handle* h, const void* d_params, const t5_batch* batch, void* d_enc_out,
@@ -155,6 +178,25 @@ T5_API int t5_encode(t5_handle* h, const void* d_params, const t5_batch* batch, 
 T5_API int t5_decode_logits(t5_handle* h, const void* d_params, const t5_batch* batch,
                      const void* d_enc_out, void* d_logits, void* d_workspace,
                      int64_t workspace_bytes, void* stream);
+
+/* Incremental decoding (the inference method applied one position at a time, "Model Implementation" section; the
+ * result at position t equals row t of t5_decode_logits on the same inputs).  One example per row (segment ids are
+ * not used).  The caller owns a cache buffer of t5_decode_cache_bytes(B, Te, Tmax) bytes that holds, per decoder
+ * layer, the self-attention keys / values of the positions decoded so far and the cross-attention keys / values.
+ *  - t5_decode_begin: resets the cache and (encoder-decoder) projects every layer's cross-attention keys / values
+ *    from d_enc_out [B, Te, d_model], the output of t5_encode; d_enc_tokens [B, Te] gives the key mask (id 0 = padding).
+ *  - t5_decode_step: position t (0, 1, 2, ... in order) of all B rows.  d_tokens [B] is the decoder INPUT at that
+ *    position (0 at t = 0, afterwards the token chosen at t - 1); writes d_logits [B, vocab] in the configured dtype
+ *    and appends the position's keys / values to the cache.  d_workspace: t5_decode_step_workspace_bytes(B) bytes.
+ * Te is ignored (may be 0) for the decoder-only architecture. */
+T5_API int t5_decode_cache_bytes(const t5_handle* h, int32_t B, int32_t Te, int32_t Tmax, int64_t* bytes);
+T5_API int t5_decode_step_workspace_bytes(const t5_handle* h, int32_t B, int64_t* bytes);
+T5_API int t5_decode_begin(t5_handle* h, const void* d_params, int32_t B, int32_t Te, int32_t Tmax,
+                           const int32_t* d_enc_tokens, const void* d_enc_out, void* d_cache, int64_t cache_bytes,
+                           void* stream);
+T5_API int t5_decode_step(t5_handle* h, const void* d_params, void* d_cache, int64_t cache_bytes, int32_t B, int32_t Te,
+                          int32_t Tmax, int32_t t, const int32_t* d_tokens, void* d_logits, void* d_workspace,
+                          int64_t workspace_bytes, void* stream);
 
 /* Reads back the status word the kernels of the last call on this workspace
  * left behind (their waits on TMA/tensor-core barriers are bounded; one that
@@ -172,6 +214,15 @@ T5_API int t5_device_status(t5_handle* h, const void* d_workspace, void* stream)
  * by the most recent step/encode/decode call on this handle. */
 T5_API int t5_profile_enable(t5_handle* h, int32_t on);
 T5_API int t5_profile_read(t5_handle* h, double ms[8], double flops[8], int64_t launches[8]);
+/* The same record launch by launch, in launch order (call it BEFORE t5_profile_read, which clears the record):
+ * what the event pair brackets, its family, the GEMM's M, N, K (0 for other kernels) and its device time.
+ * Fills at most max_records entries of `out` (host memory); *n_records receives how many exist. */
+typedef struct {
+  char what[40];
+  int32_t family, M, N, K;
+  float ms;
+} t5_profile_launch;
+T5_API int t5_profile_launches(t5_handle* h, t5_profile_launch* out, int32_t max_records, int32_t* n_records);
 T5_API int t5_launch_count(const t5_handle* h, int64_t* n);
 
 /* ---- single operations of the path, exported for element-wise parity tests ---- */

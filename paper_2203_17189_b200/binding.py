@@ -15,7 +15,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libt5b200.so")
 
-T5_ABI_VERSION = 1
+T5_ABI_VERSION = 2
 ERR_NAMES = {0: "T5_OK", -1: "T5_ERR_NULL", -2: "T5_ERR_CONFIG", -3: "T5_ERR_SHAPE", -4: "T5_ERR_ALIGN",
              -5: "T5_ERR_WORKSPACE", -6: "T5_ERR_CUDA", -7: "T5_ERR_DEVICE_TIMEOUT", -8: "T5_ERR_ARG"}
 
@@ -29,18 +29,26 @@ class t5_config(C.Structure):
                 ("max_batch", C.c_int32), ("max_enc_len", C.c_int32), ("max_dec_len", C.c_int32),
                 ("z_loss", C.c_float), ("rms_eps", C.c_float), ("attn_scale", C.c_float),
                 ("logit_scale", C.c_float),
-                ("dtype", C.c_int32), ("recompute", C.c_int32), ("flags", C.c_int32)]
+                ("dtype", C.c_int32), ("recompute", C.c_int32), ("flags", C.c_int32),
+                ("ffn_act", C.c_int32), ("untied_head", C.c_int32)]
 
 
 class t5_batch(C.Structure):
     _fields_ = [("B", C.c_int32), ("Te", C.c_int32), ("Td", C.c_int32),
                 ("d_enc_tokens", C.c_void_p), ("d_enc_segment_ids", C.c_void_p),
-                ("d_dec_targets", C.c_void_p), ("d_dec_segment_ids", C.c_void_p)]
+                ("d_dec_targets", C.c_void_p), ("d_dec_segment_ids", C.c_void_p), ("d_dec_prefix", C.c_void_p)]
+
+
+class t5_profile_launch(C.Structure):
+    _fields_ = [("what", C.c_char * 40), ("family", C.c_int32), ("M", C.c_int32), ("N", C.c_int32),
+                ("K", C.c_int32), ("ms", C.c_float)]
 
 
 EXPORTS = ["t5_create", "t5_destroy", "t5_last_error", "t5_param_count", "t5_param_tensors",
            "t5_param_manifest", "t5_workspace_bytes", "t5_init_params", "t5_train_step_fwd_bwd",
            "t5_encode", "t5_decode_logits", "t5_device_status", "t5_profile_enable", "t5_profile_read",
+           "t5_profile_launches", "t5_adamw_update", "t5_decode_cache_bytes", "t5_decode_step_workspace_bytes",
+           "t5_decode_begin", "t5_decode_step",
            "t5_launch_count", "t5_relpos_buckets", "t5_xent_zloss",
            "t5_gemm", "t5_attention", "t5_attention_backward_noalloc",
            "t5_attention_ds_scratch_bytes", "t5_attention_backward_onepass"]
@@ -73,12 +81,18 @@ def lib():
         L.t5_workspace_bytes.argtypes = [vp, C.POINTER(i64)]
         L.t5_init_params.argtypes = [vp, vp, C.c_uint64, f32, vp]
         L.t5_train_step_fwd_bwd.argtypes = [vp, vp, C.POINTER(t5_batch), vp, vp, vp, i64, vp]
+        L.t5_adamw_update.argtypes = [vp, vp, vp, vp, vp, vp, i64, f32, f32, f32, f32, f32, f32, vp]
+        L.t5_decode_cache_bytes.argtypes = [vp, i32, i32, i32, C.POINTER(i64)]
+        L.t5_decode_step_workspace_bytes.argtypes = [vp, i32, C.POINTER(i64)]
+        L.t5_decode_begin.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, i64, vp]
+        L.t5_decode_step.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, vp, i64, vp]
         L.t5_encode.argtypes = [vp, vp, C.POINTER(t5_batch), vp, vp, i64, vp]
         L.t5_decode_logits.argtypes = [vp, vp, C.POINTER(t5_batch), vp, vp, vp, i64, vp]
         L.t5_device_status.argtypes = [vp, vp, vp]
         L.t5_profile_enable.argtypes = [vp, i32]
         L.t5_profile_read.argtypes = [vp, C.POINTER(C.c_double * 8), C.POINTER(C.c_double * 8),
                                       C.POINTER(i64 * 8)]
+        L.t5_profile_launches.argtypes = [vp, C.POINTER(t5_profile_launch), i32, C.POINTER(i32)]
         L.t5_launch_count.argtypes = [vp, C.POINTER(i64)]
         L.t5_relpos_buckets.argtypes = [i32, i32, i32, i32, i32, vp, vp]
         L.t5_xent_zloss.argtypes = [i32, vp, vp, i32, i32, f32, vp, vp, vp, vp]
@@ -113,9 +127,10 @@ def _check(rc, h=None):
 
 def make_config(dims, max_batch, max_enc_len, max_dec_len, dtype, *, z_loss=1e-4, rms_eps=1e-6,
                 attn_scale=1.0, logit_scale=None, rel_buckets=32, rel_max_distance=128,
-                recompute=0, flags=0):
+                recompute=0, flags=0, ffn_act=0, untied_head=0):
     """dims: mapping with arch, n_enc_layers, n_dec_layers, d_model, n_heads, d_kv, d_ff, vocab.
-    dtype: 'f32' or 'bf16'."""
+    dtype: 'f32' or 'bf16'.  ffn_act: 0 gated GELU (tanh), 1 ReLU, 2 gated GELU (erf).  logit_scale defaults to
+    d_model^-1/2 with the tied embedding and to 1 with a separate head."""
     c = t5_config()
     c.abi_version = T5_ABI_VERSION
     for k in ("arch", "n_enc_layers", "n_dec_layers", "d_model", "n_heads", "d_kv", "d_ff", "vocab"):
@@ -123,7 +138,10 @@ def make_config(dims, max_batch, max_enc_len, max_dec_len, dtype, *, z_loss=1e-4
     c.rel_buckets, c.rel_max_distance = rel_buckets, rel_max_distance
     c.max_batch, c.max_enc_len, c.max_dec_len = max_batch, max_enc_len, max_dec_len
     c.z_loss, c.rms_eps, c.attn_scale = z_loss, rms_eps, attn_scale
-    c.logit_scale = float(dims["d_model"]) ** -0.5 if logit_scale is None else logit_scale
+    if logit_scale is None:
+        logit_scale = 1.0 if untied_head else float(dims["d_model"]) ** -0.5
+    c.logit_scale = logit_scale
+    c.ffn_act, c.untied_head = ffn_act, untied_head
     c.dtype = {"f32": 0, "bf16": 1}[dtype]
     c.recompute, c.flags = recompute, flags
     return c
@@ -191,6 +209,8 @@ class Handle:
         b.d_enc_segment_ids = None if es is None else es.data_ptr()
         b.d_dec_targets = dec.data_ptr()
         b.d_dec_segment_ids = None if ds is None else ds.data_ptr()
+        pre = batch.get("dec_prefix")
+        b.d_dec_prefix = None if pre is None else pre.data_ptr()
         return b
 
     def t5_train_step_fwd_bwd(self, params, batch, grads, loss4, workspace):
@@ -198,6 +218,30 @@ class Handle:
         _check(lib().t5_train_step_fwd_bwd(self._h, _ptr(params), C.byref(b), _ptr(grads), _ptr(loss4),
                                            _ptr(workspace), workspace.numel() * workspace.element_size(),
                                            _stream()), self._h)
+
+    def t5_adamw_update(self, params, master, m, v, grads, step, lr, beta1=0.9, beta2=0.999, eps=1e-8,
+                        weight_decay=0.0, grad_scale=1.0):
+        _check(lib().t5_adamw_update(self._h, _ptr(params), _ptr(master), _ptr(m), _ptr(v), _ptr(grads), step, lr,
+                                     beta1, beta2, eps, weight_decay, grad_scale, _stream()), self._h)
+
+    def t5_decode_cache_bytes(self, B, Te, Tmax):
+        n = C.c_int64()
+        _check(lib().t5_decode_cache_bytes(self._h, B, Te, Tmax, C.byref(n)), self._h)
+        return n.value
+
+    def t5_decode_step_workspace_bytes(self, B):
+        n = C.c_int64()
+        _check(lib().t5_decode_step_workspace_bytes(self._h, B, C.byref(n)), self._h)
+        return n.value
+
+    def t5_decode_begin(self, params, B, Te, Tmax, enc_tokens, enc_out, cache):
+        _check(lib().t5_decode_begin(self._h, _ptr(params), B, Te, Tmax, _ptr(enc_tokens), _ptr(enc_out), _ptr(cache),
+                                     cache.numel() * cache.element_size(), _stream()), self._h)
+
+    def t5_decode_step(self, params, cache, B, Te, Tmax, t, tokens, logits, workspace):
+        _check(lib().t5_decode_step(self._h, _ptr(params), _ptr(cache), cache.numel() * cache.element_size(), B, Te, Tmax,
+                                    t, _ptr(tokens), _ptr(logits), _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _stream()), self._h)
 
     def t5_encode(self, params, batch, enc_out, workspace):
         b = self._batch(batch)
@@ -219,6 +263,14 @@ class Handle:
         _check(lib().t5_profile_read(self._h, C.byref(ms), C.byref(fl), C.byref(ln)), self._h)
         names = ["gemm", "attn_fwd", "attn_bwd", "rmsnorm", "geglu", "xent", "embed", "other"]
         return {n: (ms[i], fl[i], ln[i]) for i, n in enumerate(names)}
+
+    def t5_profile_launches(self):
+        """[(what, family, M, N, K, ms)] of the profiled launches since the last t5_profile_read, in launch order"""
+        n = C.c_int32()
+        _check(lib().t5_profile_launches(self._h, None, 0, C.byref(n)), self._h)
+        buf = (t5_profile_launch * max(n.value, 1))()
+        _check(lib().t5_profile_launches(self._h, buf, n.value, C.byref(n)), self._h)
+        return [(r.what.decode(), r.family, r.M, r.N, r.K, r.ms) for r in buf[:n.value]]
 
     def t5_launch_count(self):
         n = C.c_int64()

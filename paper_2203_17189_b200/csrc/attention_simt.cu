@@ -31,7 +31,9 @@ struct P {   // plain-pointer copy of AttnArgs for the kernels
   const float* bias_delta;
   const int *code_q, *code_k;
   int B, H, Tq, Tk, causal;
+  int prefix;      // see AttnArgs::prefix: tiles are not cut at the diagonal
   float scale;
+  RowNorm rn_q, rn_k;      // row factors of dQ and of dK / dV (folded RMSNorm), see AttnArgs
 };
 
 template <typename T, int DK>
@@ -60,7 +62,7 @@ __global__ void __launch_bounds__(128) attn_fwd_kernel(P a) {
     for (int c = 0; c < C; ++c) o[qq][c] = 0.f;
   }
   int span = a.Tq + a.Tk - 1;
-  int k_end = a.causal ? min(a.Tk, q0 + 32) : a.Tk;
+  int k_end = (a.causal && !a.prefix) ? min(a.Tk, q0 + 32) : a.Tk;
   for (int k0 = 0; k0 < k_end; k0 += 32) {
     __syncthreads();
     for (int idx = tid; idx < 32 * DK; idx += 128) {
@@ -79,7 +81,7 @@ __global__ void __launch_bounds__(128) attn_fwd_kernel(P a) {
       float s = 0.f;
 #pragma unroll 8
       for (int d = 0; d < DK; ++d) s = fmaf(Qs[il * DK + d], Ks[lane * (DK + 1) + d], s);
-      bool valid = ck != 0 && ck == cq[qq] && (!a.causal || j <= i) && j < a.Tk && i < a.Tq;
+      bool valid = pair_valid(cq[qq], ck, a.causal != 0, j, i) && j < a.Tk && i < a.Tq;
       s *= a.scale;
       if (valid && a.bias_delta) s += a.bias_delta[h * span + (j - i + a.Tq - 1)];
       s = valid ? s : -INFINITY;
@@ -170,7 +172,7 @@ __global__ void __launch_bounds__(128) attn_bwd_dq_kernel(P a) {
     for (int c = 0; c < C; ++c) dq[qq][c] = 0.f;
   }
   int span = a.Tq + a.Tk - 1;
-  int k_end = a.causal ? min(a.Tk, q0 + 32) : a.Tk;
+  int k_end = (a.causal && !a.prefix) ? min(a.Tk, q0 + 32) : a.Tk;
   for (int k0 = 0; k0 < k_end; k0 += 32) {
     __syncthreads();
     for (int idx = tid; idx < 32 * DK; idx += 128) {
@@ -192,7 +194,7 @@ __global__ void __launch_bounds__(128) attn_bwd_dq_kernel(P a) {
         s = fmaf(Qs[il * DK + d], Ks[lane * (DK + 1) + d], s);
         dp = fmaf(dOs[il * DK + d], Vs[lane * (DK + 1) + d], dp);
       }
-      bool valid = ck != 0 && ck == cq[qq] && (!a.causal || j <= i) && j < a.Tk && i < a.Tq &&
+      bool valid = pair_valid(cq[qq], ck, a.causal != 0, j, i) && j < a.Tk && i < a.Tq &&
                    lse[qq] != -INFINITY;
       s *= a.scale;
       if (valid && a.bias_delta) s += a.bias_delta[h * span + (j - i + a.Tq - 1)];
@@ -211,9 +213,10 @@ __global__ void __launch_bounds__(128) attn_bwd_dq_kernel(P a) {
   for (int qq = 0; qq < 8; ++qq) {
     int i = q0 + warp * 8 + qq;
     if (i >= a.Tq) continue;
+    const float f = a.scale * rn_factor(a.rn_q, (int64_t)b * a.Tq + i);
 #pragma unroll
     for (int c = 0; c < C; ++c)
-      dQ[(int64_t)(b * a.Tq + i) * a.lddq + h * DK + lane + 32 * c] = from_f<T>(a.scale * dq[qq][c]);
+      dQ[(int64_t)(b * a.Tq + i) * a.lddq + h * DK + lane + 32 * c] = from_f<T>(f * dq[qq][c]);
   }
   if (want_db) {
     __syncthreads();
@@ -258,7 +261,7 @@ __global__ void __launch_bounds__(128) attn_bwd_dkv_kernel(P a) {
     for (int c = 0; c < C; ++c) dk[kk][c] = dv[kk][c] = 0.f;
   }
   int span = a.Tq + a.Tk - 1;
-  int q_begin = a.causal ? k0 : 0;     // k0 is a multiple of 32: queries before it see none of these keys
+  int q_begin = (a.causal && !a.prefix) ? k0 : 0;     // k0 is a multiple of 32: queries before it see none of these keys
   for (int q0 = q_begin; q0 < a.Tq; q0 += 32) {
     __syncthreads();
     for (int idx = tid; idx < 32 * DK; idx += 128) {
@@ -287,7 +290,7 @@ __global__ void __launch_bounds__(128) attn_bwd_dkv_kernel(P a) {
         s = fmaf(Qs[lane * (DK + 1) + d], Ks[jl * DK + d], s);
         dp = fmaf(dOs[lane * (DK + 1) + d], Vs[jl * DK + d], dp);
       }
-      bool valid = ck[kk] != 0 && ck[kk] == cq && (!a.causal || j <= i) && j < a.Tk && i < a.Tq &&
+      bool valid = pair_valid(cq, ck[kk], a.causal != 0, j, i) && j < a.Tk && i < a.Tq &&
                    lse != -INFINITY;
       s *= a.scale;
       if (valid && a.bias_delta) s += a.bias_delta[h * span + (j - i + a.Tq - 1)];
@@ -309,10 +312,11 @@ __global__ void __launch_bounds__(128) attn_bwd_dkv_kernel(P a) {
   for (int kk = 0; kk < 8; ++kk) {
     int j = k0 + warp * 8 + kk;
     if (j >= a.Tk) continue;
+    const float f = rn_factor(a.rn_k, (int64_t)b * a.Tk + j);
 #pragma unroll
     for (int c = 0; c < C; ++c) {
-      dK[(int64_t)(b * a.Tk + j) * a.lddk + h * DK + lane + 32 * c] = from_f<T>(a.scale * dk[kk][c]);
-      dV[(int64_t)(b * a.Tk + j) * a.lddv + h * DK + lane + 32 * c] = from_f<T>(dv[kk][c]);
+      dK[(int64_t)(b * a.Tk + j) * a.lddk + h * DK + lane + 32 * c] = from_f<T>(f * a.scale * dk[kk][c]);
+      dV[(int64_t)(b * a.Tk + j) * a.lddv + h * DK + lane + 32 * c] = from_f<T>(f * dv[kk][c]);
     }
   }
 }
@@ -325,6 +329,8 @@ P to_p(const AttnArgs& a) {
   p.O32 = a.O32; p.ldo32 = a.ldo32;
   p.bias_delta = a.bias_delta; p.code_q = a.code_q; p.code_k = a.code_k; p.B = a.B; p.H = a.H;
   p.Tq = a.Tq; p.Tk = a.Tk; p.causal = a.causal; p.scale = a.scale;
+  p.rn_q = a.rn_q; p.rn_k = a.rn_k;
+  p.prefix = a.prefix;
   return p;
 }
 

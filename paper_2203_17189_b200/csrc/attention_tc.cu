@@ -49,6 +49,8 @@ struct TcParams {
   int* status;
   int bias_far;              // see AttnArgs::bias_far
   int packed;                // see AttnArgs::packed
+  int prefix;                // see AttnArgs::prefix: no tile is cut off at the diagonal
+  RowNorm rn_q, rn_k;        // see AttnArgs: row factors of dQ and of dK / dV
 };
 
 
@@ -135,7 +137,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
   const int tid = threadIdx.x, warp = tid >> 5;
   const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * 128;
   int n_kt = (p.Tk + 63) / 64;
-  if (p.causal) n_kt = min(n_kt, (q0 + 127) / 64 + 1);
+  if (p.causal && !p.prefix) n_kt = min(n_kt, (q0 + 127) / 64 + 1);
   constexpr uint32_t kTmemCols = DK == 64 ? 128 : 256;
 
   if (tid == 0) {
@@ -210,7 +212,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
   int n_act = n_kt;
   if (p.packed) {
     int* rng = tiles_s + n_tiles_cap;                  // [8]: (lo, hi) of each warp's rows
-    int lo = cq ? cq : 0x7fffffff, hi = cq;
+    const int cqs = cq & ~T5_PREFIX_BIT;               // segment part of the code
+    int lo = cqs ? cqs : 0x7fffffff, hi = cqs;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
@@ -230,7 +233,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
       const int t = base + (lane >> 4);
       int klo = 0x7fffffff, khi = 0;
       if (t < n_kt) {
-        const int4 c = *reinterpret_cast<const int4*>(codes_s + t * 64 + (lane & 15) * 4);
+        int4 c = *reinterpret_cast<const int4*>(codes_s + t * 64 + (lane & 15) * 4);
+        c.x &= ~T5_PREFIX_BIT; c.y &= ~T5_PREFIX_BIT; c.z &= ~T5_PREFIX_BIT; c.w &= ~T5_PREFIX_BIT;
         klo = min(min(c.x ? c.x : 0x7fffffff, c.y ? c.y : 0x7fffffff), min(c.z ? c.z : 0x7fffffff, c.w ? c.w : 0x7fffffff));
         khi = ::max(::max(c.x, c.y), ::max(c.z, c.w));
       }
@@ -287,7 +291,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
           for (int jj = 0; jj < 32; ++jj) {
             int j = k0 + c * 32 + jj;
             int ck = codes_s[j];
-            bool valid = ck != 0 && ck == cq && (!p.causal || j <= i);
+            bool valid = pair_valid(cq, ck, p.causal != 0, j, i);
             sc[c][jj] = valid ? sc[c][jj] : -INFINITY;
           }
         }
@@ -439,7 +443,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
   const int tid = threadIdx.x, warp = tid >> 5, row = tid & 127, half = tid >> 7, quad = warp & 3;
   const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * 128;
   int n_kt = (p.Tk + 63) / 64;
-  if (p.causal) n_kt = min(n_kt, (q0 + 127) / 64 + 1);
+  if (p.causal && !p.prefix) n_kt = min(n_kt, (q0 + 127) / 64 + 1);
   constexpr uint32_t kTmemCols = 256;
   const bool want_db = p.dbias_delta != nullptr;
 
@@ -557,7 +561,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
           if (!FAST) {
             int j = k0 + c * 32 + jj;
             int ck = codes_s[j];
-            bool valid = ck != 0 && ck == cq && (!p.causal || j <= i) && lse2 != -INFINITY;
+            bool valid = pair_valid(cq, ck, p.causal != 0, j, i) && lse2 != -INFINITY;
             pr = valid ? pr : 0.f;
           }
           ds[jj] = pr * (__uint_as_float(rp[jj]) - dl);
@@ -625,6 +629,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
   if (ok) {
     tc_fence_after();
     bf16* drow = (bf16*)p.out0 + (int64_t)(b * p.Tq + i) * p.ld0 + h * DK + half * (DK / 2);
+    const float fq = row_in ? p.scale * rn_factor(p.rn_q, (int64_t)b * p.Tq + i) : 0.f;
 #pragma unroll
     for (int c = 0; c < DK / 64; ++c) {
       uint32_t r[32];
@@ -634,10 +639,10 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_const
 #pragma unroll
         for (int d = 0; d < 32; d += 8) {
           uint4 v;
-          v.x = pack_bf16(p.scale * __uint_as_float(r[d]), p.scale * __uint_as_float(r[d + 1]));
-          v.y = pack_bf16(p.scale * __uint_as_float(r[d + 2]), p.scale * __uint_as_float(r[d + 3]));
-          v.z = pack_bf16(p.scale * __uint_as_float(r[d + 4]), p.scale * __uint_as_float(r[d + 5]));
-          v.w = pack_bf16(p.scale * __uint_as_float(r[d + 6]), p.scale * __uint_as_float(r[d + 7]));
+          v.x = pack_bf16(fq * __uint_as_float(r[d]), fq * __uint_as_float(r[d + 1]));
+          v.y = pack_bf16(fq * __uint_as_float(r[d + 2]), fq * __uint_as_float(r[d + 3]));
+          v.z = pack_bf16(fq * __uint_as_float(r[d + 4]), fq * __uint_as_float(r[d + 5]));
+          v.w = pack_bf16(fq * __uint_as_float(r[d + 6]), fq * __uint_as_float(r[d + 7]));
           *reinterpret_cast<uint4*>(drow + c * 32 + d) = v;
         }
       }
@@ -714,7 +719,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
   const int tid = threadIdx.x, warp = tid >> 5, row = tid & 127, half = tid >> 7, quad = warp & 3;
   const int b = blockIdx.z, h = blockIdx.y, k0 = blockIdx.x * 128;
   const int n_qt = (p.Tq + 63) / 64;
-  const int t_begin = p.causal ? k0 / 64 : 0;          // queries before k0 see none of these keys
+  const int t_begin = (p.causal && !p.prefix) ? k0 / 64 : 0;          // queries before k0 see none of these keys
   constexpr uint32_t kTmemCols = DK == 64 ? 256 : 512;
 
   if (tid == 0) {
@@ -835,7 +840,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
             if (!FAST) {
               int q = qb + c * 32 + ii;
               int cq = codes_s[q];
-              bool valid = ck != 0 && ck == cq && (!p.causal || j <= q) && lse2 != -INFINITY;
+              bool valid = pair_valid(cq, ck, p.causal != 0, j, q) && lse2 != -INFINITY;
               pr = valid ? pr : 0.f;
             }
             pt[ii] = pr;
@@ -887,6 +892,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
     bf16* krow = (bf16*)p.out0 + (int64_t)(b * p.Tk + j) * p.ld0 + h * DK + half * (DK / 2);
     bf16* vrow = (bf16*)p.out1 + (int64_t)(b * p.Tk + j) * p.ld1 + h * DK + half * (DK / 2);
     const bool any = t_begin < n_qt;
+    const float fv = row_in ? rn_factor(p.rn_k, (int64_t)b * p.Tk + j) : 0.f, fk = p.scale * fv;
 #pragma unroll
     for (int c = 0; c < DK / 64; ++c) {
       uint32_t rv[32], rk[32];
@@ -903,15 +909,15 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
 #pragma unroll
         for (int d = 0; d < 32; d += 8) {
           uint4 v;
-          v.x = pack_bf16(__uint_as_float(rv[d]), __uint_as_float(rv[d + 1]));
-          v.y = pack_bf16(__uint_as_float(rv[d + 2]), __uint_as_float(rv[d + 3]));
-          v.z = pack_bf16(__uint_as_float(rv[d + 4]), __uint_as_float(rv[d + 5]));
-          v.w = pack_bf16(__uint_as_float(rv[d + 6]), __uint_as_float(rv[d + 7]));
+          v.x = pack_bf16(fv * __uint_as_float(rv[d]), fv * __uint_as_float(rv[d + 1]));
+          v.y = pack_bf16(fv * __uint_as_float(rv[d + 2]), fv * __uint_as_float(rv[d + 3]));
+          v.z = pack_bf16(fv * __uint_as_float(rv[d + 4]), fv * __uint_as_float(rv[d + 5]));
+          v.w = pack_bf16(fv * __uint_as_float(rv[d + 6]), fv * __uint_as_float(rv[d + 7]));
           *reinterpret_cast<uint4*>(vrow + c * 32 + d) = v;
-          v.x = pack_bf16(p.scale * __uint_as_float(rk[d]), p.scale * __uint_as_float(rk[d + 1]));
-          v.y = pack_bf16(p.scale * __uint_as_float(rk[d + 2]), p.scale * __uint_as_float(rk[d + 3]));
-          v.z = pack_bf16(p.scale * __uint_as_float(rk[d + 4]), p.scale * __uint_as_float(rk[d + 5]));
-          v.w = pack_bf16(p.scale * __uint_as_float(rk[d + 6]), p.scale * __uint_as_float(rk[d + 7]));
+          v.x = pack_bf16(fk * __uint_as_float(rk[d]), fk * __uint_as_float(rk[d + 1]));
+          v.y = pack_bf16(fk * __uint_as_float(rk[d + 2]), fk * __uint_as_float(rk[d + 3]));
+          v.z = pack_bf16(fk * __uint_as_float(rk[d + 4]), fk * __uint_as_float(rk[d + 5]));
+          v.w = pack_bf16(fk * __uint_as_float(rk[d + 6]), fk * __uint_as_float(rk[d + 7]));
           *reinterpret_cast<uint4*>(krow + c * 32 + d) = v;
         }
       }
@@ -1038,7 +1044,7 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.z, h = blockIdx.y, k0 = blockIdx.x * 128;
   const int n_qt = (p.Tq + 63) / 64;
-  const int t_begin = p.causal ? k0 / 64 : 0;          // queries before k0 see none of these keys
+  const int t_begin = (p.causal && !p.prefix) ? k0 / 64 : 0;          // queries before k0 see none of these keys
   const int n = n_qt - t_begin;                        // tiles this CTA walks
   constexpr uint32_t kTmemCols = DK == 64 ? 256 : 512;
   constexpr uint32_t kColS = 0, kColDP = 64, kColDV = 128, kColDK = 128 + DK;
@@ -1166,6 +1172,8 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
     const int quad = warp & 3, half = warp >> 2, row = quad * 32 + lane;
     const int j = k0 + row;
     const int ck = j < p.Tk ? p.code_k[b * p.Tk + j] : 0;
+    // row factor of this key's dK / dV rows (folded RMSNorm), fetched now so that the epilogue does not wait for it
+    const float fv_row = j < p.Tk ? rn_factor(p.rn_k, (int64_t)b * p.Tk + j) : 0.f;
     {
       // The per-CTA tables are filled here, by the softmax warps alone and behind their own barrier: the loads
       // and the first S^T / dP^T MMAs of the other two warps run meanwhile.  One batched fill of the four tables
@@ -1238,7 +1246,7 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
               if (!FAST) {
                 int q = qq0 + ii;
                 int cqv = codes_s[q];
-                bool valid = ck != 0 && ck == cqv && (!p.causal || j <= q) && lse2 != -INFINITY;
+                bool valid = pair_valid(cqv, ck, p.causal != 0, j, q) && lse2 != -INFINITY;
                 pr = valid ? pr : 0.f;
               }
               pt[ii] = pr;
@@ -1320,6 +1328,7 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
       // tensor map.  dV uses the P^T / dS^T tiles, dK the dS^T tile (d_kv 64) or the Q / dO ring (d_kv 128).
       unsigned char* tV = smem + L::kP0;
       unsigned char* tK = DK == 64 ? smem + L::kDS0 : smem + L::kQD0;
+      const float fv = fv_row, fk = p.scale * fv;
 #pragma unroll
       for (int c = 0; c < DK / 32; ++c) {
         const int col = half * (DK / 2) + c * 16;          // this pass's 16 output columns
@@ -1338,15 +1347,15 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
         for (int q8 = 0; q8 < 2; ++q8) {
           const int d = q8 * 8;
           uint4 v;
-          v.x = pack_bf16(__uint_as_float(rv[d]), __uint_as_float(rv[d + 1]));
-          v.y = pack_bf16(__uint_as_float(rv[d + 2]), __uint_as_float(rv[d + 3]));
-          v.z = pack_bf16(__uint_as_float(rv[d + 4]), __uint_as_float(rv[d + 5]));
-          v.w = pack_bf16(__uint_as_float(rv[d + 6]), __uint_as_float(rv[d + 7]));
+          v.x = pack_bf16(fv * __uint_as_float(rv[d]), fv * __uint_as_float(rv[d + 1]));
+          v.y = pack_bf16(fv * __uint_as_float(rv[d + 2]), fv * __uint_as_float(rv[d + 3]));
+          v.z = pack_bf16(fv * __uint_as_float(rv[d + 4]), fv * __uint_as_float(rv[d + 5]));
+          v.w = pack_bf16(fv * __uint_as_float(rv[d + 6]), fv * __uint_as_float(rv[d + 7]));
           store_swizzled_16B(tV + chunk * 16384, row, piece0 + q8, v);
-          v.x = pack_bf16(p.scale * __uint_as_float(rk[d]), p.scale * __uint_as_float(rk[d + 1]));
-          v.y = pack_bf16(p.scale * __uint_as_float(rk[d + 2]), p.scale * __uint_as_float(rk[d + 3]));
-          v.z = pack_bf16(p.scale * __uint_as_float(rk[d + 4]), p.scale * __uint_as_float(rk[d + 5]));
-          v.w = pack_bf16(p.scale * __uint_as_float(rk[d + 6]), p.scale * __uint_as_float(rk[d + 7]));
+          v.x = pack_bf16(fk * __uint_as_float(rk[d]), fk * __uint_as_float(rk[d + 1]));
+          v.y = pack_bf16(fk * __uint_as_float(rk[d + 2]), fk * __uint_as_float(rk[d + 3]));
+          v.z = pack_bf16(fk * __uint_as_float(rk[d + 4]), fk * __uint_as_float(rk[d + 5]));
+          v.w = pack_bf16(fk * __uint_as_float(rk[d + 6]), fk * __uint_as_float(rk[d + 7]));
           store_swizzled_16B(tK + chunk * 16384, row, piece0 + q8, v);
         }
       }
@@ -1417,7 +1426,7 @@ attn_bwd_dq_ds_tc_kernel(const __grid_constant__ CUtensorMap mds, const __grid_c
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * 128;
   int n_kt = (p.Tk + 63) / 64;
-  if (p.causal) n_kt = min(n_kt, (q0 + 127) / 64 + 1);
+  if (p.causal && !p.prefix) n_kt = min(n_kt, (q0 + 127) / 64 + 1);
   constexpr uint32_t kTmemCols = DK;
 
   if (tid == 0) {
@@ -1471,6 +1480,7 @@ attn_bwd_dq_ds_tc_kernel(const __grid_constant__ CUtensorMap mds, const __grid_c
   } else {
     // epilogue: warps 2-5; warp w may touch tensor-memory lanes 32 (w % 4) ..
     const int quad = warp & 3, row = quad * 32 + lane, i = q0 + row;
+    const float fq = i < p.Tq ? p.scale * rn_factor(p.rn_q, (int64_t)b * p.Tq + i) : 0.f;      // before the wait
     ok = mbar_wait(done, 0, abort_flag, p.status, 53);
     if (ok) {
       tc_fence_after();
@@ -1490,10 +1500,10 @@ attn_bwd_dq_ds_tc_kernel(const __grid_constant__ CUtensorMap mds, const __grid_c
 #pragma unroll
           for (int d = 0; d < 32; d += 8) {
             uint4 v;
-            v.x = pack_bf16(p.scale * __uint_as_float(r[d]), p.scale * __uint_as_float(r[d + 1]));
-            v.y = pack_bf16(p.scale * __uint_as_float(r[d + 2]), p.scale * __uint_as_float(r[d + 3]));
-            v.z = pack_bf16(p.scale * __uint_as_float(r[d + 4]), p.scale * __uint_as_float(r[d + 5]));
-            v.w = pack_bf16(p.scale * __uint_as_float(r[d + 6]), p.scale * __uint_as_float(r[d + 7]));
+            v.x = pack_bf16(fq * __uint_as_float(r[d]), fq * __uint_as_float(r[d + 1]));
+            v.y = pack_bf16(fq * __uint_as_float(r[d + 2]), fq * __uint_as_float(r[d + 3]));
+            v.z = pack_bf16(fq * __uint_as_float(r[d + 4]), fq * __uint_as_float(r[d + 5]));
+            v.w = pack_bf16(fq * __uint_as_float(r[d + 6]), fq * __uint_as_float(r[d + 7]));
             *reinterpret_cast<uint4*>(drow + c * 32 + d) = v;
           }
         }
@@ -1529,6 +1539,8 @@ TcParams base_params(const AttnArgs& a, int* status) {
   p.packed = a.packed;
   p.dbias_delta = a.dbias_delta; p.B = a.B; p.H = a.H; p.Tq = a.Tq; p.Tk = a.Tk; p.causal = a.causal;
   p.scale = a.scale; p.status = status;
+  p.rn_q = a.rn_q; p.rn_k = a.rn_k;
+  p.prefix = a.prefix;
   return p;
 }
 

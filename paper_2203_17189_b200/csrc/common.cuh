@@ -46,8 +46,31 @@ __host__ __device__ inline int bucket_of(const BucketSpec& s, int rel) {
   return off + s.me + q;
 }
 
+// Position codes: 0 for padding, else the segment id (1 if unpacked); in a prefix LM the positions of the fully
+// visible prefix also carry T5_PREFIX_BIT.  Query (code cq, position i) may attend key (ck, j) iff both belong to
+// the same segment and, when causal, j <= i or both lie in the prefix.
+#define T5_PREFIX_BIT 0x40000000
+__host__ __device__ __forceinline__ bool pair_valid(int cq, int ck, bool causal, int j, int i) {
+  const int sk = ck & ~T5_PREFIX_BIT;
+  return sk != 0 && (cq & ~T5_PREFIX_BIT) == sk && (!causal || j <= i || ((cq & ck) & T5_PREFIX_BIT) != 0);
+}
+
 // Builds the thresholds; returns false if the parameters are unsupported.
 bool build_bucket_spec(int bidirectional, int num_buckets, int max_distance, BucketSpec* out);
+
+// ---------------------------------------------------------------------------
+// RMSNorm folded into the GEMMs around it.  y = x (mean(x^2) + eps)^-1/2 g feeds a projection y W^T; here the
+// kernel that produces the residual row x also writes xg = x * g (operand dtype) and adds the row's sum of
+// squares into ssq[row]; the projection runs on xg and its epilogue multiplies row m of the product by
+// (ssq[m] / d + eps)^-1/2.  A RowNorm names such a statistics vector; ssq == NULL means "no factor".
+// ---------------------------------------------------------------------------
+struct RowNorm {
+  const float* ssq;   // [rows] sum over the d columns of x^2, float32
+  float inv_d, eps;
+};
+__device__ __forceinline__ float rn_factor(const RowNorm& r, int64_t row) {
+  return r.ssq ? rsqrtf(r.ssq[row] * r.inv_d + r.eps) : 1.f;
+}
 
 // ---------------------------------------------------------------------------
 // Launchers.  `dtype` selects float / bf16 storage for "T" tensors; all
@@ -69,6 +92,12 @@ struct GemmArgs {
   //                    da = d(hg) * b * gelu'(a) and db = d(hg) * gelu(a).
   int epi; void* aux; int ld_aux; int F;
   int pair;                               // 1: 256 x 256 tiles on CTA pairs (cta_group::2) where M, N >= 256
+  // RMSNorm fold, consumer side: row m of the product (epi 0, 1) or of d(hg) (epi 2) is multiplied by rn's factor
+  RowNorm rn;
+  // RMSNorm fold, producer side (float32 output with a residual addend only): besides D = alpha A B + resid the
+  // epilogue writes xg[m, n] = D[m, n] * g_next[n] in the operand dtype and adds sum_n D[m, n]^2 of its columns
+  // into ssq_out[m] (zeroed by the caller before the GEMM)
+  void* xg_out; int ld_xg; const void* g_next; float* ssq_out;
   int* sk_flags;                          // optional: >= 160 zeroed ints; lets the tcgen05 kernel split the
                                           // tiles of a partial last wave along K over all SMs (float32 output)
 };
@@ -107,9 +136,15 @@ struct AttnArgs {
   // one pass over the scores (dK, dV and a bf16 copy of dS^T in this buffer) and takes dQ from the stored dS
   void* ds_scratch = nullptr;
   int64_t ds_bytes = 0;
+  // backward only: rows of dQ are multiplied by rn_q's factor, rows of dK and dV by rn_k's (the RMSNorm fold of
+  // the projections that made q, k, v wants their gradients scaled that way; NULL statistics = factor 1)
+  RowNorm rn_q = {nullptr, 0.f, 0.f}, rn_k = {nullptr, 0.f, 0.f};
   // non-zero: rows may hold several segments (packed examples).  The tcgen05 forward then leaves out key tiles whose
   // range of position codes does not meet the range of the CTA's query rows; 0 skips that bookkeeping.
   int packed = 0;
+  // non-zero: causal attention whose position codes may carry T5_PREFIX_BIT (prefix LM): keys ahead of a query can
+  // be valid, so the kernels walk every tile instead of stopping at the diagonal
+  int prefix = 0;
 };
 int64_t attn_tc_ds_scratch_bytes(int B, int H, int Tq, int Tk);
 bool attn_tc_onepass_supported(const AttnArgs& a);   // the backward will take the one-pass route
@@ -121,30 +156,47 @@ cudaError_t attn_fwd_tc(const AttnArgs& a, int* d_status, cudaStream_t st);
 cudaError_t attn_bwd_tc(const AttnArgs& a, int* d_status, cudaStream_t st);
 
 // element-wise / row kernels
+// dec_prefix (optional 0/1 flags): flagged positions get T5_PREFIX_BIT in their code and loss weight 0
 cudaError_t launch_prep(const int* enc_tok, const int* enc_seg, const int* dec_tgt, const int* dec_seg,
-                        int B, int Te, int Td, int* enc_code, int* dec_code, int* dec_in,
-                        int* W_int, float* W_f, cudaStream_t st);
-cudaError_t launch_embed_gather(int dtype, const void* E, const int* tok, float* X, int n_tok, int d,
-                                cudaStream_t st);
+                        const int* dec_prefix, int B, int Te, int Td, int* enc_code, int* dec_code, int* dec_in,
+                        float* dec_w, int* W_int, float* W_f, cudaStream_t st);
+cudaError_t launch_pad_codes(const int* tok, int* code, int n, cudaStream_t st);      // code = tok != 0
+cudaError_t launch_set_column(int* p, int ld, int col, int rows, int value, cudaStream_t st);
+// X[t] = E[tok[t]] (float32); with g != NULL also XG[t] = X[t] * g (dtype T) and ssq[t] = sum X[t]^2
+cudaError_t launch_embed_gather(int dtype, const void* E, const int* tok, float* X, const void* g, void* XG,
+                                float* ssq, int n_tok, int d, cudaStream_t st);
 cudaError_t launch_embed_scatter_add(const int* tok, const float* dX, float* dE, int n_tok, int d,
                                      cudaStream_t st);
 cudaError_t launch_rmsnorm_fwd(int dtype, const float* X, const void* g, void* Y, float* rstd,
                                int rows, int d, float eps, cudaStream_t st);
-// dX_out = (dX_in ? dX_in : 0) + rmsnorm_bwd(dy); writes float32 dX_out and a T copy dXb (if non-NULL).
-// dy is float32 if dy_f32 else T.  dg (float32 [d]) is OVERWRITTEN; partial: scratch [n_part*d].
-cudaError_t launch_rmsnorm_bwd(int dtype, const void* dy, int dy_f32, const float* X, const float* rstd,
+// Backward of the folded RMSNorm.  t = gradient wrt xg = x * g, i.e. (row factor r) * (gradient wrt the normed
+// activations): what the data-gradient GEMM of a projection leaves when its incoming gradient rows carry the
+// factor r.  dx = g t - x (r^2 / d) sum_k (t g x)_k;  dg = sum_rows t x.
+// dX_out = (dX_in ? dX_in : 0) + dx; writes float32 dX_out and a T copy dXb (if non-NULL).
+// t is float32 if t_f32 else T.  dg (float32 [d]) is OVERWRITTEN; partial: scratch [n_part*d].
+cudaError_t launch_rmsnorm_bwd(int dtype, const void* t, int t_f32, const float* X, RowNorm rn,
                                const void* g, const float* dX_in, float* dX_out, void* dXb, float* dg,
                                float* partial, int rows, int d, cudaStream_t st);
+// XG = X * g (dtype T): recomputes the operand copy of a residual row block
+cudaError_t launch_scale_cols(int dtype, const float* X, const void* g, void* XG, int rows, int d, cudaStream_t st);
 int rmsnorm_bwd_parts(int rows);
-cudaError_t launch_geglu_fwd(int dtype, const void* h, void* hg, int rows, int F, cudaStream_t st);
-cudaError_t launch_geglu_bwd(int dtype, const void* dhg, const void* h, void* dh, int rows, int F,
+// FFN non-linearity.  act 0 / 2: h [rows, 2F] = [a | b], hg = gelu(a) * b (tanh form / exact erf form);
+// act 1: h [rows, F], hg = relu(h).
+cudaError_t launch_geglu_fwd(int dtype, int act, const void* h, void* hg, int rows, int F, cudaStream_t st);
+// its backward (dh has h's shape); rows of dh are multiplied by rn's factor
+cudaError_t launch_geglu_bwd(int dtype, int act, const void* dhg, const void* h, void* dh, int rows, int F, RowNorm rn,
                              cudaStream_t st);
-cudaError_t launch_xent(int dtype, void* logits, const int* targets, int rows, int V, float z,
-                        const float* W, double* sums, float* lse, cudaStream_t st);
+// weights: per-row loss weights (NULL: 1 where the target is not padding); rows of the gradient written over the
+// logits are multiplied by rn's factor
+cudaError_t launch_xent(int dtype, void* logits, const int* targets, const float* weights, int rows, int V, float z,
+                        const float* W, double* sums, float* lse, RowNorm rn, cudaStream_t st);
 cudaError_t launch_finalize_loss(const double* sums, const float* W, float* loss4, cudaStream_t st);
 cudaError_t launch_fill_normal(int dtype, void* p, int64_t n, int64_t flat_offset, uint64_t seed,
                                float stddev, float mean, cudaStream_t st);
-cudaError_t launch_round_bf16(float* p, int64_t n, cudaStream_t st);   // in place: float -> nearest bf16 -> float
+// AdamW on elements [0, n) of the given pointers (n a multiple of 4); see t5_adamw_update
+cudaError_t launch_adamw(int dtype, void* params, float* master, float* m, float* v, const float* g, int64_t n,
+                         float lr, float b1, float b2, float eps, float wd, float gscale, float bc1, float bc2,
+                         cudaStream_t st);
 cudaError_t launch_cast_f32_to(int dtype, const float* src, void* dst, int64_t n, cudaStream_t st);
 // bias tables
 cudaError_t launch_relbias_expand(int dtype, const BucketSpec& spec, const void* table, int H, int Tq,

@@ -11,7 +11,8 @@ template <typename T, typename TD, bool AK, bool BK>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(int M, int N, int K, float alpha,
                                                         const T* __restrict__ A, int lda,
                                                         const T* __restrict__ B, int ldb, TD* D, int ldd,
-                                                        const float* resid, int ldr, int accumulate) {
+                                                        const float* resid, int ldr, int accumulate, RowNorm rn,
+                                                        T* xg_out, int ld_xg, const T* g_next, float* ssq_out) {
   __shared__ float As[TK][TM + 4];
   __shared__ float Bs[TK][TN + 4];
   int tid = threadIdx.x;
@@ -61,16 +62,23 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(int M, int N, int K, flo
   for (int i = 0; i < 4; ++i) {
     int gm = m0 + ty * 4 + i;
     if (gm >= M) continue;
+    const float arow = alpha * rn_factor(rn, gm);      // folded RMSNorm: factor of the product's row
+    float ss = 0.f;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       int gn = n0 + tx * 4 + j;
       if (gn >= N) continue;
-      float v = alpha * acc[i][j];
+      float v = arow * acc[i][j];
       if (resid != nullptr) v += resid[(int64_t)gm * ldr + gn];
       TD* dp = D + (int64_t)gm * ldd + gn;
       if (accumulate) v += to_f(*dp);
       *dp = from_f<TD>(v);
+      if (xg_out != nullptr) {      // producer side of the fold: operand copy x * g and the row's sum of squares
+        xg_out[(int64_t)gm * ld_xg + gn] = from_f<T>(v * to_f(g_next[gn]));
+        ss += v * v;
+      }
     }
+    if (xg_out != nullptr) atomicAdd(ssq_out + gm, ss);
   }
 }
 
@@ -81,7 +89,8 @@ cudaError_t launch(const GemmArgs& g, cudaStream_t st) {
 #define GO(AK, BK)                                                                                   \
   gemm_simt_kernel<T, TD, AK, BK><<<grid, 256, 0, st>>>(g.M, g.N, g.K, g.alpha, (const T*)g.A, g.lda, \
                                                         (const T*)g.B, g.ldb, (TD*)g.D, g.ldd, g.resid, \
-                                                        g.ldr, g.accumulate)
+                                                        g.ldr, g.accumulate, g.rn, (T*)g.xg_out, g.ld_xg,    \
+                                                        (const T*)g.g_next, g.ssq_out)
   if (g.a_kmajor && g.b_kmajor) GO(true, true);
   else if (g.a_kmajor) GO(true, false);
   else if (g.b_kmajor) GO(false, true);

@@ -45,7 +45,18 @@ struct Params {
   // (a partial wave) are cut along K into gridDim.x equal ranges of k-blocks.  sk_rem = 0 turns it off.
   int sk_full, sk_rem;
   int* sk_flags;      // [sk_rem], zeroed: counts the epilogue warps of the storing segment that are done
+  // RMSNorm fold (see GemmArgs): row factor of the product; operand copy + sum of squares of the new residual rows
+  RowNorm rn;
+  bf16* xg_out;
+  int ld_xg;
+  const bf16* g_next;
+  float* ssq_out;
 };
+
+// alpha times the RMSNorm factor of the accumulator row this thread holds (tensor-memory lane = row)
+__device__ __forceinline__ float row_alpha(const Params& p, int row) {
+  return (p.rn.ssq != nullptr && row < p.M) ? p.alpha * rsqrtf(p.rn.ssq[row] * p.rn.inv_d + p.rn.eps) : p.alpha;
+}
 
 // One unit of work of a CTA: k-blocks [kb0, kb1) of a tile.
 //   kind 0: the whole tile;  1: the segment that reaches the tile's last k-block (it stores, then raises
@@ -98,29 +109,70 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
   tm = first + r % gsz;
   tn = r / gsz;
 }
+__device__ __forceinline__ void store_bf16x4(bf16* d, float4 v) {
+  __nv_bfloat162 b0 = __floats2bfloat162_rn(v.x, v.y), b1 = __floats2bfloat162_rn(v.z, v.w);
+  uint2 o;
+  o.x = *reinterpret_cast<uint32_t*>(&b0);
+  o.y = *reinterpret_cast<uint32_t*>(&b1);
+  *reinterpret_cast<uint2*>(d) = o;
+}
+__device__ __forceinline__ float4 load_bf16x4(const bf16* p) {
+  uint2 u = *reinterpret_cast<const uint2*>(p);
+  return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                     __uint_as_float(u.y & 0xffff0000u));
+}
 // Epilogue of one 128-row x BN-column accumulator tile for one warp (rows quad*32 .. +31 of the tile).
 // Each thread holds one accumulator row; going through a per-warp shared-memory tile turns the stores (and the
 // loads of the float32 addend) into 128-byte row segments instead of 32 scattered pieces.
 // Chunks (32 columns each) [c_begin, c_end) of the tile are this warp's share.
+// What an epilogue warp can fetch before its tile's accumulator is ready (while it waits for the MMAs): the row's
+// RMSNorm factor, the first chunk of the float32 addend and the first chunk's norm scales.
+struct EpiPre {
+  float arow;
+  float4 add0[8];
+  float4 gn0;
+};
+__device__ __forceinline__ const float* epi_addend(const Params& p, bool add_atomic) {
+  return (!p.out_f32 || add_atomic) ? nullptr : (p.resid ? p.resid : (p.accumulate ? (const float*)p.D : nullptr));
+}
+__device__ __forceinline__ void epi_fetch_addend(const Params& p, const float* addend, int m0, int n0, int quad, int lane,
+                                                 int c, float4 (&dst)[8]) {
+  const int rr0 = lane >> 3, col = n0 + c * 32 + (lane & 7) * 4;
+  const int ld_add = p.resid ? p.ldr : p.ldd;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = m0 + quad * 32 + i * 4 + rr0;
+    dst[i] = (addend && row < p.M && col < p.N) ? *reinterpret_cast<const float4*>(addend + (int64_t)row * ld_add + col)
+                                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+}
+__device__ __forceinline__ float4 epi_fetch_gn(const Params& p, int n0, int lane, int c) {
+  const int col = n0 + c * 32 + (lane & 7) * 4;
+  return (p.xg_out != nullptr && col < p.N) ? load_bf16x4(p.g_next + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+}
+__device__ __forceinline__ void epi_prefetch(const Params& p, int m0, int n0, int quad, int lane, bool add_atomic,
+                                             int c_begin, EpiPre& pre) {
+  pre.arow = row_alpha(p, m0 + quad * 32 + lane);
+  if (p.epi == 0) {
+    epi_fetch_addend(p, epi_addend(p, add_atomic), m0, n0, quad, lane, c_begin, pre.add0);
+    pre.gn0 = epi_fetch_gn(p, n0, lane, c_begin);
+  }
+}
+
 template <int BN>
 __device__ __forceinline__ void store_tile(const Params& p, float* tbuf, uint32_t tacc, int m0, int n0, int quad,
-                                           int lane, bool add_atomic, int c_begin = 0, int c_end = BN / 32) {
+                                           int lane, bool add_atomic, const EpiPre& pre, int c_begin = 0,
+                                           int c_end = BN / 32) {
   const int rr0 = lane >> 3, cc = (lane & 7) * 4;
-  // float32 addend (residual input, or D itself when accumulating), fetched one chunk ahead of its use
-  const float* addend = (!p.out_f32 || add_atomic) ? nullptr
-                                                    : (p.resid ? p.resid : (p.accumulate ? (const float*)p.D : nullptr));
-  const int ld_add = p.resid ? p.ldr : p.ldd;
-  float4 add_next[8];
-  auto fetch_addend = [&](int c, float4 (&dst)[8]) {
-    const int col = n0 + c * 32 + cc;
+  const float arow = pre.arow;
+  const bool fold_out = p.xg_out != nullptr && !add_atomic;      // also write x * g and the rows' sums of squares
+  float ss[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  // float32 addend (residual input, or D itself when accumulating) and the next norm's scales, fetched one chunk
+  // ahead of their use (the first chunk's before the accumulator was ready)
+  const float* addend = epi_addend(p, add_atomic);
+  float4 add_next[8], gn_next = pre.gn0;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int row = m0 + quad * 32 + i * 4 + rr0;
-      dst[i] = (addend && row < p.M && col < p.N) ? *reinterpret_cast<const float4*>(addend + (int64_t)row * ld_add + col)
-                                                    : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-  };
-  fetch_addend(c_begin, add_next);
+  for (int i = 0; i < 8; ++i) add_next[i] = pre.add0[i];
 #pragma unroll 1
   for (int c = c_begin; c < c_end; ++c) {
     const int col0 = n0 + c * 32;
@@ -128,16 +180,20 @@ __device__ __forceinline__ void store_tile(const Params& p, float* tbuf, uint32_
     float4 add_cur[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) add_cur[i] = add_next[i];
+    const float4 gn = gn_next;
     uint32_t r[32];
     tmem_ld_32x32b_x32(tacc + c * 32, r);
     tmem_wait_ld_dep(r);
 #pragma unroll
     for (int j = 0; j < 8; ++j)
       *reinterpret_cast<float4*>(tbuf + lane * 36 + j * 4) =
-          make_float4(p.alpha * __uint_as_float(r[4 * j]), p.alpha * __uint_as_float(r[4 * j + 1]),
-                      p.alpha * __uint_as_float(r[4 * j + 2]), p.alpha * __uint_as_float(r[4 * j + 3]));
+          make_float4(arow * __uint_as_float(r[4 * j]), arow * __uint_as_float(r[4 * j + 1]),
+                      arow * __uint_as_float(r[4 * j + 2]), arow * __uint_as_float(r[4 * j + 3]));
     __syncwarp();
-    if (addend && c + 1 < c_end) fetch_addend(c + 1, add_next);       // in flight while this chunk is stored
+    if (c + 1 < c_end) {                                               // in flight while this chunk is stored
+      if (addend) epi_fetch_addend(p, addend, m0, n0, quad, lane, c + 1, add_next);
+      if (fold_out) gn_next = epi_fetch_gn(p, n0, lane, c + 1);
+    }
     const int col = col0 + cc;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -152,6 +208,10 @@ __device__ __forceinline__ void store_tile(const Params& p, float* tbuf, uint32_
         } else if (p.out_f32) {
           v.x += add_cur[i].x; v.y += add_cur[i].y; v.z += add_cur[i].z; v.w += add_cur[i].w;
           *reinterpret_cast<float4*>((float*)p.D + (int64_t)row * p.ldd + col) = v;
+          if (fold_out) {
+            store_bf16x4(p.xg_out + (int64_t)row * p.ld_xg + col, make_float4(v.x * gn.x, v.y * gn.y, v.z * gn.z, v.w * gn.w));
+            ss[i] += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+          }
         } else {
           bf16* d = (bf16*)p.D + (int64_t)row * p.ldd + col;
           __nv_bfloat162 b0 = __floats2bfloat162_rn(v.x, v.y), b1 = __floats2bfloat162_rn(v.z, v.w);
@@ -164,6 +224,18 @@ __device__ __forceinline__ void store_tile(const Params& p, float* tbuf, uint32_
     }
     __syncwarp();                          // the tile is rewritten by the next chunk
   }
+  if (fold_out) {
+    // the eight lanes that share a row (same lane >> 3) add up their columns' squares; one atomic per row
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      float t = ss[i];
+      t += __shfl_xor_sync(0xffffffffu, t, 1);
+      t += __shfl_xor_sync(0xffffffffu, t, 2);
+      t += __shfl_xor_sync(0xffffffffu, t, 4);
+      const int row = m0 + quad * 32 + i * 4 + rr0;
+      if ((lane & 7) == 0 && row < p.M) atomicAdd(p.ssq_out + row, t);
+    }
+  }
 }
 
 // ---- gated-GELU epilogues (tanh approximation through the hardware tanh; outputs are bf16)
@@ -173,18 +245,6 @@ __device__ __forceinline__ void gelu_both_fast(float u, float& g, float& dg) {
   asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(c * (u + a * u * u2)));
   g = 0.5f * u * (1.f + t);
   dg = 0.5f * (1.f + t) + 0.5f * u * (1.f - t * t) * c * (1.f + 3.f * a * u2);
-}
-__device__ __forceinline__ void store_bf16x4(bf16* d, float4 v) {
-  __nv_bfloat162 b0 = __floats2bfloat162_rn(v.x, v.y), b1 = __floats2bfloat162_rn(v.z, v.w);
-  uint2 o;
-  o.x = *reinterpret_cast<uint32_t*>(&b0);
-  o.y = *reinterpret_cast<uint32_t*>(&b1);
-  *reinterpret_cast<uint2*>(d) = o;
-}
-__device__ __forceinline__ float4 load_bf16x4(const bf16* p) {
-  uint2 u = *reinterpret_cast<const uint2*>(p);
-  return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
-                     __uint_as_float(u.y & 0xffff0000u));
 }
 // one accumulator chunk (32 columns of this thread's row) -> the warp's coalesced layout (8 x float4 per lane)
 __device__ __forceinline__ void transpose_chunk(float* tbuf, int lane, const uint32_t (&r)[32], float alpha, float4 (&v)[8]) {
@@ -201,7 +261,7 @@ __device__ __forceinline__ void transpose_chunk(float* tbuf, int lane, const uin
 }
 // forward: accumulator columns [0,128) = a, [128,256) = b of feature block tn; writes h = [a | b] and hg = gelu(a) b
 __device__ __forceinline__ void store_tile_geglu_fwd(const Params& p, float* tbuf, uint32_t tacc, int m0, int tn, int quad,
-                                                     int lane, int c_begin = 0, int c_end = 4) {
+                                                     int lane, float arow, int c_begin = 0, int c_end = 4) {
   const int rr0 = lane >> 3, cc = (lane & 7) * 4;
   bf16* H = (bf16*)p.D;
   bf16* HG = (bf16*)p.aux;
@@ -213,8 +273,8 @@ __device__ __forceinline__ void store_tile_geglu_fwd(const Params& p, float* tbu
     tmem_wait_ld_dep(ra);
     tmem_wait_ld_dep(rb);
     float4 va[8], vb[8];
-    transpose_chunk(tbuf, lane, ra, p.alpha, va);
-    transpose_chunk(tbuf, lane, rb, p.alpha, vb);
+    transpose_chunk(tbuf, lane, ra, arow, va);
+    transpose_chunk(tbuf, lane, rb, arow, vb);
     const int col = tn * 128 + c * 32 + cc;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -236,8 +296,8 @@ __device__ __forceinline__ void store_tile_geglu_fwd(const Params& p, float* tbu
 // backward: the accumulator is d(hg); aux = h = [a | b]; writes dh = [d(hg) b gelu'(a) | d(hg) gelu(a)]
 template <int BN>
 __device__ __forceinline__ void store_tile_geglu_bwd(const Params& p, float* tbuf, uint32_t tacc, int m0, int n0, int quad,
-                                                     int lane, int c_begin = 0, int c_end = BN / 32) {
-  const int rr0 = lane >> 3, cc = (lane & 7) * 4;
+                                                     int lane, float arow, int c_begin = 0, int c_end = BN / 32) {
+  const int rr0 = lane >> 3, cc = (lane & 7) * 4;      // arow: d(hg) rows carry the norm factor, da and db are linear in it
   const bf16* Hh = (const bf16*)p.aux;
   bf16* DH = (bf16*)p.D;
 #pragma unroll 1
@@ -256,7 +316,7 @@ __device__ __forceinline__ void store_tile_geglu_bwd(const Params& p, float* tbu
       bv[i] = in ? load_bf16x4(Hh + (int64_t)row * p.ld_aux + p.F + col) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     float4 v[8];
-    transpose_chunk(tbuf, lane, r, p.alpha, v);
+    transpose_chunk(tbuf, lane, r, arow, v);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int row = m0 + quad * 32 + i * 4 + rr0;
@@ -415,6 +475,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int m0 = tm * BM, n0 = tn * BN;
       const int ab = it & 1;
       const uint32_t aph = (it >> 1) & 1;
+      EpiPre pre;
+      epi_prefetch(p, m0, n0, quad, lane, w.kind == 2, 0, pre);
       ok = mbar_wait(&tfull[ab], aph, abort_flag, p.status, 4);
       if (ok && w.kind == 2) {
         // an earlier K-segment of a split tile: the segment that stores must be done first
@@ -435,7 +497,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       tc_fence_after();
       const bool add_atomic = w.kind == 2;
       store_tile<BN>(p, reinterpret_cast<float*>(smem + S::kEpiOffset) + quad * (32 * 36),
-                     tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16), m0, n0, quad, lane, add_atomic);
+                     tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16), m0, n0, quad, lane, add_atomic, pre);
       if (w.kind == 1) {          // publish this warp's part of the stored tile to the adding segments
         __threadfence();
         __syncwarp();
@@ -466,16 +528,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // the heavier epilogues (gated-GELU backward, float32 residual) ran at the pace of one warp's instruction latencies,
 // longer than the tile's MMAs; a second warp per scheduler hides them.  The transpose buffers of the extra warps
 // take the room of the sixth stage.
-constexpr int kThreads2 = 384;
+constexpr int kThreads2 = 384;          // 4 + kEpiWarps2 warps
+constexpr int kEpiWarps2 = 8;
 constexpr int STAGES2 = 5;
 struct Smem2 {
   static constexpr int kABytes = 128 * BK * 2, kBBytes = 128 * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kBarOffset = STAGES2 * kStageBytes;
   static constexpr int kEpiOffset = kBarOffset + 256;
-  static constexpr int kEpiBytes = 8 * 32 * 36 * 4;
+  static constexpr int kEpiBytes = kEpiWarps2 * 32 * 36 * 4;
   static constexpr int kTotal = kEpiOffset + kEpiBytes + 1024;
 };
+static_assert(Smem2::kTotal <= 227 * 1024, "shared memory of the CTA-pair kernel");
 
 template <bool A_MN, bool B_MN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
@@ -499,10 +563,12 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   const int k_blocks = (p.K + BK - 1) / BK;
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   constexpr uint32_t kTmemCols = 512;
+  // epilogue warps: n_epi / 4 per tensor-memory lane quarter, each with a share of the tile's eight 32-column chunks
+  const int n_epi = (int)(blockDim.x >> 5) - 4, n_col_groups = n_epi >> 2;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES2; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 16); }  // 8 warps of each CTA
+    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 2 * n_epi); }  // the epilogue warps of both CTAs
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -584,7 +650,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
-    const int quad = warp & 3, ew = warp - 4, ch = ew >> 2;      // ch: which half of the tile's columns
+    const int quad = warp & 3, ew = warp - 4, ch = ew >> 2;      // ch: which share of the tile's columns
+    const int c0 = ch * 8 / n_col_groups, c1 = (ch + 1) * 8 / n_col_groups;
+    // gated-GELU forward: four chunk pairs (a and b of the same features), split over at most two groups
+    const int g0 = ch < 2 ? ch * 2 : 4, g1 = ch < 2 ? ch * 2 + 2 : 4;
     int it = 0;
     bool ok = true;
     WorkIter wi(p, k_blocks, pair, n_pairs);
@@ -595,12 +664,14 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const int m0 = tm * 256 + (int)rank * 128, n0 = tn * 256;
       const int ab = it & 1;
       const uint32_t aph = (it >> 1) & 1;
+      EpiPre pre;
+      epi_prefetch(p, m0, n0, quad, lane, w.kind == 2, c0, pre);
       ok = mbar_wait(&tfull[ab], aph, abort_flag, p.status, 9);
       if (ok && w.kind == 2) {
         // an earlier K-segment of a split tile: the storing pair (16 epilogue warps) must be done first
         volatile int* flag = p.sk_flags + w.flag;
         long long t0 = clock64();
-        while (*flag < 16) {
+        while (*flag < 2 * n_epi) {
           if (clock64() - t0 > kWaitCycles) {
             if (p.status) atomicCAS(p.status, 0, 10);
             ok = false;
@@ -615,9 +686,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       tc_fence_after();
       float* tb = reinterpret_cast<float*>(smem + S::kEpiOffset) + ew * (32 * 36);
       const uint32_t tacc = tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16);
-      if (p.epi == 1) store_tile_geglu_fwd(p, tb, tacc, m0, tn, quad, lane, ch * 2, ch * 2 + 2);
-      else if (p.epi == 2) store_tile_geglu_bwd<BN>(p, tb, tacc, m0, n0, quad, lane, ch * 4, ch * 4 + 4);
-      else store_tile<BN>(p, tb, tacc, m0, n0, quad, lane, w.kind == 2, ch * 4, ch * 4 + 4);
+      if (p.epi == 1) store_tile_geglu_fwd(p, tb, tacc, m0, tn, quad, lane, pre.arow, g0, g1);
+      else if (p.epi == 2) store_tile_geglu_bwd<BN>(p, tb, tacc, m0, n0, quad, lane, pre.arow, c0, c1);
+      else store_tile<BN>(p, tb, tacc, m0, n0, quad, lane, w.kind == 2, pre, c0, c1);
       if (w.kind == 1) {
         __threadfence();
         __syncwarp();
@@ -684,6 +755,7 @@ cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& 
   p.resid = g.resid; p.ldr = g.ldr; p.accumulate = g.accumulate;
   p.tiles_m = (g.M + BM - 1) / BM; p.tiles_n = (g.N + BN - 1) / BN; p.status = status;
   p.epi = 0; p.aux = nullptr; p.ld_aux = 0; p.F = 0;
+  p.rn = g.rn; p.xg_out = (bf16*)g.xg_out; p.ld_xg = g.ld_xg; p.g_next = (const bf16*)g.g_next; p.ssq_out = g.ssq_out;
   int tiles = p.tiles_m * p.tiles_n;
   int grid = tiles < g_num_sms ? tiles : g_num_sms;
   p.sk_full = 0; p.sk_rem = 0; p.sk_flags = nullptr;
@@ -692,7 +764,7 @@ cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& 
   // split the tiles of a partial last wave along K when that wave would leave a good part of the GPU idle
   // (measured: pays only for long K and after at least one full wave; short-K tiles lose more in the extra
   // atomic epilogues than the idle SMs cost)
-  if (g.sk_flags && g.out_f32 && rem > 0 && k_blocks >= 128 && tiles >= g_num_sms && g_num_sms <= 160 &&
+  if (g.sk_flags && g.out_f32 && !g.xg_out && rem > 0 && k_blocks >= 128 && tiles >= g_num_sms && g_num_sms <= 160 &&
       (g_num_sms - rem) * 8 > g_num_sms * (tiles / g_num_sms + 1)) {
     grid = g_num_sms;
     p.sk_full = tiles / g_num_sms; p.sk_rem = rem; p.sk_flags = g.sk_flags;
@@ -714,12 +786,13 @@ cudaError_t launch2(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap&
   p.resid = g.resid; p.ldr = g.ldr; p.accumulate = g.accumulate;
   p.tiles_m = (g.M + 255) / 256; p.tiles_n = g.epi == 1 ? g.F / 128 : (g.N + 255) / 256; p.status = status;
   p.epi = g.epi; p.aux = g.aux; p.ld_aux = g.ld_aux; p.F = g.F;
+  p.rn = g.rn; p.xg_out = (bf16*)g.xg_out; p.ld_xg = g.ld_xg; p.g_next = (const bf16*)g.g_next; p.ssq_out = g.ssq_out;
   p.sk_full = 0; p.sk_rem = 0; p.sk_flags = nullptr;
   int tiles = p.tiles_m * p.tiles_n;
   int pairs = g_num_sms / 2;
   const int k_blocks = (g.K + BK - 1) / BK, rem = tiles % pairs;
   // long-K float32-output GEMMs: split the tiles of a partial last wave along K over all pairs
-  if (g.epi == 0 && g.sk_flags && g.out_f32 && rem > 0 && k_blocks >= 128 && tiles >= pairs && pairs <= 160 &&
+  if (g.epi == 0 && g.sk_flags && g.out_f32 && !g.xg_out && rem > 0 && k_blocks >= 128 && tiles >= pairs && pairs <= 160 &&
       (pairs - rem) * 8 > pairs * (tiles / pairs + 1)) {
     p.sk_full = tiles / pairs; p.sk_rem = rem; p.sk_flags = g.sk_flags;
   } else if (tiles < pairs) {
@@ -766,6 +839,9 @@ bool gemm_tc_supported(const GemmArgs& g) {
   if (g.N % 4) return false;
   if (g.resid && (!al16(g.resid) || g.ldr % 4)) return false;
   if (g.accumulate && !g.out_f32) return false;
+  if (g.xg_out && (!g.out_f32 || !g.resid || g.accumulate || !g.g_next || !g.ssq_out || !al16(g.xg_out) ||
+                   ((uintptr_t)g.g_next & 7) || g.ld_xg % 4))
+    return false;
   return tc::get_encode() != nullptr;
 }
 

@@ -3,7 +3,7 @@ checks: conversion between the library's flat parameter buffer and the
 oracle's named tensors, and the comparison metrics."""
 import numpy as np
 
-DENSE_SUFFIXES = (".q", ".k", ".v", ".o", ".wi0", ".wi1", ".wo")
+DENSE_SUFFIXES = (".q", ".k", ".v", ".o", ".wi0", ".wi1", ".wo", "lm_head")
 
 
 def is_dense(name):
