@@ -511,7 +511,7 @@ void attn_args(Ctx& cx, const AttnWs& a, const AttnGeom& gm, bool cross, AttnArg
   t.O = a.ctx; t.ldo = I; t.lse = a.lse; t.O32 = a.ctx32; t.ldo32 = I;
   t.B = cx.B; t.H = c.n_heads; t.Tq = gm.Tq; t.Tk = gm.Tk; t.dk = c.d_kv;
   t.code_q = gm.code_q; t.code_k = gm.code_k; t.causal = gm.causal;
-  t.bias_delta = gm.bias; t.scale = c.attn_scale;
+  t.bias_delta = gm.bias; t.scale = c.attn_scale; t.bias_far = gm.far;
   t.packed = cx.packed;
   t.prefix = gm.prefix;
 }
