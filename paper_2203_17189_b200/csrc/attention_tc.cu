@@ -924,7 +924,7 @@ struct KvfLayout {
   static constexpr int kBarBytes = 128;
   static int bytes(int Tq, bool want_db) {
     int tqp = (Tq + 63) / 64 * 64;
-    return kMisc + (tqp + 128) * 4 + 3 * tqp * 4 + (want_db ? (tqp + 128) * 4 : 0) + kBarBytes + 1024 + 64;
+    return kMisc + (tqp + 128) * 4 + 3 * tqp * 4 + (want_db ? (tqp + 128) * 4 : 0) + (tqp / 64 + 4) * 4 + kBarBytes + 1024 + 64;
   }
 };
 
@@ -958,19 +958,21 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
   float* dl_s = lse_s + tqp;                          // [tqp]
   int* codes_s = (int*)(dl_s + tqp);                  // [tqp] query codes
   float* dbias_s = (float*)(codes_s + tqp);           // [tqp + 128], entry (key row - query + tqp)
-  KvfBars* bars = (KvfBars*)(((uintptr_t)(dbias_s + (want_db ? tqp + 128 : 0)) + 15) & ~(uintptr_t)15);
+  int* qt_s = (int*)(dbias_s + (want_db ? tqp + 128 : 0));      // [tqp / 64 + 2] query tiles this CTA walks (packed rows)
+  KvfBars* bars = (KvfBars*)(((uintptr_t)(qt_s + tqp / 64 + 4) + 15) & ~(uintptr_t)15);
   volatile int* abort_flag = &bars->abort_flag;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.z, h = blockIdx.y, k0 = blockIdx.x * 128;
   const int n_qt = (p.Tq + 63) / 64;
   const int t_begin = (p.causal && !p.prefix) ? k0 / 64 : 0;          // queries before k0 see none of these keys
-  const int n = n_qt - t_begin;                        // tiles this CTA walks
+  int n = n_qt - t_begin;                              // tiles this CTA walks (fewer on packed rows, see below)
+  auto tile_of = [&](int i) { return p.packed ? qt_s[i] : t_begin + i; };
   constexpr uint32_t kTmemCols = DK == 64 ? 256 : 512;
   constexpr uint32_t kColS = 0, kColDP = 64, kColDV = 128, kColDK = 128 + DK;
 
   auto load_qd = [&](int i) {
-    const int st = i % NST, t = t_begin + i;
+    const int st = i % NST, t = tile_of(i);
     unsigned char* base = smem + L::kQD0 + st * L::kStage;
     mbar_arrive_expect_tx(&bars->qd_full[st], L::kStage);
 #pragma unroll
@@ -989,6 +991,8 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
     mbar_init(&bars->acc, 1);
     bars->abort_flag = 0;
     fence_barrier_init();
+  }
+  auto first_loads = [&]() {
     if (n > 0) {
       mbar_arrive_expect_tx(&bars->kv, 2 * L::kKVBytes);
 #pragma unroll
@@ -998,6 +1002,15 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
       }
       for (int i = 0; i < NST && i < n; ++i) load_qd(i);
     }
+  };
+  if (!p.packed) {
+    if (tid == 9 * 32) first_loads();
+  } else {
+    // packed rows: query tiles whose 128-query block shares no segment with this CTA's keys are left out (the dQ
+    // kernel applies the same rule, so the regions of the dS scratch that stay unwritten are never read)
+    n = packed_tile_list<kKvfThreads>(p.code_k + (int64_t)b * p.Tk, p.Tk, k0, p.code_q + (int64_t)b * p.Tq, p.Tq, t_begin,
+                                      n_qt, qt_s, tid);
+    if (tid == 9 * 32) first_loads();
   }
   if (warp == 8) tmem_alloc(&bars->tmem, kTmemCols);
   const int span = p.Tq + p.Tk - 1;
@@ -1013,7 +1026,7 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
       for (int i = 0; i < n && ok; ++i) {
         ok = mbar_wait_relaxed(&bars->p_full, i & 1, abort_flag, p.status, 41);
         if (!ok) break;
-        tma_store_3d(&mds, smem + L::kDS0, (t_begin + i) * 64, k0, b * p.H + h);
+        tma_store_3d(&mds, smem + L::kDS0, tile_of(i) * 64, k0, b * p.H + h);
         bulk_commit_group();
         if (i + NST < n) {    // the reload goes out before the store's read is waited for: its latency is the longer one
           ok = mbar_wait_relaxed(&bars->qd_free[i % NST], (i / NST) & 1, abort_flag, p.status, 42);
@@ -1126,7 +1139,7 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
     unsigned char* tP = smem + L::kP0;
     unsigned char* tD = smem + L::kDS0;
     for (int i = 0; i < n && ok; ++i) {
-      const int qb = (t_begin + i) * 64;
+      const int qb = tile_of(i) * 64;
       const uint32_t par = i & 1;
       ok = __all_sync(0xffffffffu, mbar_wait_relaxed(&bars->s_full, par, abort_flag, p.status, 46));
       if (!ok) break;
@@ -1328,7 +1341,8 @@ struct DqsLayout {
   static constexpr int kABytes = 2 * 8192, kBBytes = 64 * DK * 2;
   static constexpr int kStage = kABytes + kBBytes;
   static constexpr int kBar = kStages * kStage;
-  static constexpr int kTotal = kBar + 256 + 1024;
+  static constexpr int kList = kBar + 256;                       // key tiles this CTA walks (packed rows): up to 130 ints
+  static constexpr int kTotal = kList + 1024 + 1024;
 };
 
 template <int DK>
@@ -1348,6 +1362,8 @@ attn_bwd_dq_ds_tc_kernel(const __grid_constant__ CUtensorMap mds, const __grid_c
   int n_kt = (p.Tk + 63) / 64;
   if (p.causal && !p.prefix) n_kt = min(n_kt, (q0 + 127) / 64 + 1);
   constexpr uint32_t kTmemCols = DK;
+  int* kt_s = (int*)(smem + L::kList);
+  auto tile_of = [&](int u) { return p.packed ? kt_s[u] : u; };
 
   if (tid == 0) {
     for (int s = 0; s < NST; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -1355,6 +1371,9 @@ attn_bwd_dq_ds_tc_kernel(const __grid_constant__ CUtensorMap mds, const __grid_c
     *abort_flag = 0;
     fence_barrier_init();
   }
+  // packed rows: the key tiles the dK / dV kernel left out for these queries hold nothing it stored
+  if (p.packed)
+    n_kt = packed_tile_list<192>(p.code_q + (int64_t)b * p.Tq, p.Tq, q0, p.code_k + (int64_t)b * p.Tk, p.Tk, 0, n_kt, kt_s, tid);
   if (warp == 1) tmem_alloc(tmem_holder, kTmemCols);
   tc_fence_before();
   __syncthreads();
@@ -1365,9 +1384,9 @@ attn_bwd_dq_ds_tc_kernel(const __grid_constant__ CUtensorMap mds, const __grid_c
   if (warp == 0) {
     if (lane == 0) {
       int issued = 0;
-      for (int t = 0; t < n_kt; ++t) {
-        const int s = t % NST;
-        if (!mbar_wait(&empty[s], ((t / NST) & 1) ^ 1, abort_flag, p.status, 51)) { ok = false; break; }
+      for (int u = 0; u < n_kt; ++u) {
+        const int s = u % NST, t = tile_of(u);
+        if (!mbar_wait(&empty[s], ((u / NST) & 1) ^ 1, abort_flag, p.status, 51)) { ok = false; break; }
         unsigned char* sa = smem + s * L::kStage;
         mbar_arrive_expect_tx(&full[s], L::kStage);
         tma_load_3d(sa, &mds, q0, t * 64, b * p.H + h, &full[s]);
@@ -1385,7 +1404,7 @@ attn_bwd_dq_ds_tc_kernel(const __grid_constant__ CUtensorMap mds, const __grid_c
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc(128, DK, true, true);
-      for (int t = 0; t < n_kt; ++t) {
+      for (int t = 0; t < n_kt; ++t) {      // t counts the tiles walked, not key positions
         const int s = t % NST;
         if (!mbar_wait(&full[s], (t / NST) & 1, abort_flag, p.status, 52)) { ok = false; break; }
         tc_fence_after();

@@ -85,6 +85,60 @@ struct Bars {
   int abort_flag;
 };
 
+
+// Packed rows: which 64-row tiles of the "other" side (queries for a key block, keys for a query block) can hold a
+// valid pair with this CTA's 128 "own" rows.  A pair is valid only if both positions carry the same non-zero
+// segment code, so a 128-row block of the other side whose range of non-zero codes does not meet the range of the
+// own rows holds none; its two tiles are left out.  The rule is taken per pair of 128-row blocks so that the kernel
+// that walks key blocks and the kernel that walks query blocks leave out exactly the same (query, key) regions (the
+// second one reads what the first one stored).
+// Writes the kept tiles of [t_begin, t_end) (t_begin even) in increasing order to list_s and returns their number.
+// list_s: shared memory, t_end + 2 ints.  Every thread of the CTA (NT of them) must call; contains barriers.
+template <int NT>
+__device__ int packed_tile_list(const int* own_codes, int T_own, int own0, const int* other_codes, int T_other,
+                                int t_begin, int t_end, int* list_s, int tid) {
+  const int warp = tid >> 5, lane = tid & 31;
+  int* own_rng = list_s + t_end;
+  auto range128 = [&](const int* codes, int T, int r0, int& lo, int& hi) {
+    lo = 0x7fffffff; hi = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int r = r0 + lane + 32 * k;
+      const int c = r < T ? (codes[r] & ~T5_PREFIX_BIT) : 0;
+      if (c) { lo = min(lo, c); hi = ::max(hi, c); }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = ::max(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+  };
+  int lo, hi;
+  if (warp == 0) {
+    range128(own_codes, T_own, own0, lo, hi);
+    if (lane == 0) { own_rng[0] = lo; own_rng[1] = hi; }
+  }
+  __syncthreads();
+  const int slo = own_rng[0], shi = own_rng[1];
+  for (int pb = t_begin / 2 + warp; 2 * pb < t_end; pb += NT / 32) {
+    range128(other_codes, T_other, pb * 128, lo, hi);
+    const int act = (shi > 0 && hi > 0 && hi >= slo && lo <= shi) ? 1 : 0;
+    if (lane == 0) {
+      list_s[2 * pb] = act;
+      if (2 * pb + 1 < t_end) list_s[2 * pb + 1] = act;
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {      // compaction in place: the write position never passes the read position
+    int n = 0;
+    for (int t = t_begin; t < t_end; ++t)
+      if (list_s[t]) list_s[n++] = t;
+    own_rng[0] = n;
+  }
+  __syncthreads();
+  return own_rng[0];
+}
+
 // ----------------------------------------------------------------------------- host side
 // 3-D view [B][T][cols] of a row-major token matrix with row stride ld; box = [1][rows][64 cols]
 bool make_map3(CUtensorMap* m, const void* base, int cols, int T, int B, int ld, int box_rows) {

@@ -1382,6 +1382,7 @@ int t5_attention_backward_onepass(int32_t B, int32_t H, int32_t Tq, int32_t Tk, 
   a.bias_delta = d_bias_delta; a.scale = scale; a.dO = d_do; a.lddo = lddo; a.dQ = d_dq; a.dK = d_dk; a.dV = d_dv;
   a.lddq = lddq; a.lddk = lddk; a.lddv = lddv; a.delta = d_delta; a.dbias_delta = d_dbias_delta;
   a.bias_far = bias_far; a.ds_scratch = d_ds_scratch; a.ds_bytes = ds_scratch_bytes;
+  a.packed = 1;      // the codes may describe packed rows: keep the tile-skipping bookkeeping on
   if (!attn_tc_supported(a) || !attn_tc_onepass_supported(a)) return T5_ERR_ARG;
   cudaError_t e = attn_bwd_tc(a, nullptr, (cudaStream_t)stream);
   return e == cudaSuccess ? T5_OK : T5_ERR_CUDA;
