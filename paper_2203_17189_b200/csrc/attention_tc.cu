@@ -191,6 +191,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
     const bool fast = tcode > 0 && __all_sync(0xffffffffu, cq == tcode) &&
                       (!p.causal || k0 + 63 <= q0 + (warp << 5));          // warp-uniform: no mask needed
     const float* brow = bias_s + (k0 - tid + 127);
+    // the whole tile lies where the bias no longer depends on the distance (saturated bucket): one value, no loads
+    const bool flat = has_bias && p.bias_far > 0 && (k0 - (q0 + 127) >= p.bias_far || q0 - (k0 + 63) >= p.bias_far);
     float sc[2][32];
     {
       uint32_t r[2][32];
@@ -199,7 +201,11 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         tmem_wait_ld_dep(r[c]);
-        if (has_bias) {
+        if (flat) {
+          const float b0 = brow[0];
+#pragma unroll
+          for (int jj = 0; jj < 32; ++jj) sc[c][jj] = fmaf(__uint_as_float(r[c][jj]), sc2, b0);
+        } else if (has_bias) {
 #pragma unroll
           for (int jj = 0; jj < 32; ++jj) sc[c][jj] = fmaf(__uint_as_float(r[c][jj]), sc2, brow[c * 32 + jj]);
         } else {
@@ -1163,8 +1169,11 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
           if (lane == 0) mbar_arrive(&bars->s_free);
         }
         float pt[16], ds[16];
+        // bias_c: 0 none, 1 per distance, 2 one value for the whole pass (saturated bucket)
         auto compute = [&](auto fast_c, auto bias_c) {
-          constexpr bool FAST = decltype(fast_c)::value, BIAS = decltype(bias_c)::value;
+          constexpr bool FAST = decltype(fast_c)::value;
+          constexpr int BIAS = decltype(bias_c)::value;
+          const float bflat = BIAS == 2 ? brow[0] : 0.f;
 #pragma unroll
           for (int i4 = 0; i4 < 4; ++i4) {
             const float4 l4 = *reinterpret_cast<const float4*>(lse_s + qq0 + i4 * 4);
@@ -1174,7 +1183,8 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
               const int ii = i4 * 4 + e;
               const float lse2 = e == 0 ? l4.x : e == 1 ? l4.y : e == 2 ? l4.z : l4.w;
               const float dlq = e == 0 ? d4.x : e == 1 ? d4.y : e == 2 ? d4.z : d4.w;
-              float sv = BIAS ? fmaf(__uint_as_float(rs[ii]), sc2, brow[-ii]) : __uint_as_float(rs[ii]) * sc2;
+              float sv = BIAS == 1 ? fmaf(__uint_as_float(rs[ii]), sc2, brow[-ii])
+                                   : BIAS == 2 ? fmaf(__uint_as_float(rs[ii]), sc2, bflat) : __uint_as_float(rs[ii]) * sc2;
               float pr = ex2_approx(sv - lse2);
               if (!FAST) {
                 int q = qq0 + ii;
@@ -1187,10 +1197,17 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
             }
           }
         };
+        using B0 = std::integral_constant<int, 0>;
+        using B1 = std::integral_constant<int, 1>;
+        using B2 = std::integral_constant<int, 2>;
+        const int kk0b = k0 + quad * 32;                 // this pass: keys [kk0b, kk0b + 32) x queries [qq0, qq0 + 16)
+        const bool flat = has_bias && p.bias_far > 0 && (kk0b - (qq0 + 15) >= p.bias_far || qq0 - (kk0b + 31) >= p.bias_far);
         if (fast) {
-          if (has_bias) compute(std::true_type{}, std::true_type{}); else compute(std::true_type{}, std::false_type{});
+          if (flat) compute(std::true_type{}, B2{});
+          else if (has_bias) compute(std::true_type{}, B1{});
+          else compute(std::true_type{}, B0{});
         } else {
-          if (has_bias) compute(std::false_type{}, std::true_type{}); else compute(std::false_type{}, std::false_type{});
+          if (has_bias) compute(std::false_type{}, B1{}); else compute(std::false_type{}, B0{});
         }
         if (want_db) {
           const int kk0 = k0 + quad * 32;                  // this pass: 32 keys x 16 queries
