@@ -297,6 +297,28 @@ T5_API int t5_attention_backward_onepass(
     void* d_dv, int32_t lddv, float* d_delta, float* d_dbias_delta, int32_t bias_far, void* d_ds_scratch,
     int64_t ds_scratch_bytes, void* stream);
 
+/* Status word for the kernel-level entry points (t5_attention,
+ * t5_attention_backward_onepass, t5_attention_backward_noalloc, t5_gemm): they
+ * have no workspace whose first word could carry it.  d_status: device int32,
+ * zeroed by the caller, or NULL to switch reporting off (the default).  A
+ * tensor-core kernel whose bounded wait on a TMA / MMA barrier runs out writes
+ * its code there (first one wins), abandons its tile and returns normally; the
+ * outputs of that call are then incomplete.  The pointer is process-wide and
+ * read at launch time; the caller owns the word and reads it after
+ * synchronising the stream.  ("Model Implementation" section: the methods a
+ * model exposes must report failure to the training loop; the paper names no
+ * mechanism.)  Returns T5_OK. */
+T5_API int t5_kernel_status_word(int32_t* d_status);
+
+/* Exercises the give-up path of the kernels' bounded waits without hanging
+ * anything: one small CTA waits, with the same wait routine the tensor-core
+ * kernels use, on a barrier that nothing ever arrives at.  After limit_cycles
+ * SM cycles (1 .. 4e9) the wait gives up, writes code 99 into *d_status (device
+ * int32, zeroed by the caller) and the kernel returns in the ordinary way; the
+ * context stays usable.  No memory traffic, no tensor memory.
+ * T5_ERR_NULL / T5_ERR_ARG for bad arguments. */
+T5_API int t5_selftest_bounded_wait(int32_t* d_status, int64_t limit_cycles, void* stream);
+
 /* Attention backward without caller-provided scratch.  The paper has no
  * counterpart; this exists for callers that cannot allocate device memory:
  * code in a region where cudaMalloc is illegal or must be avoided, plug-ins

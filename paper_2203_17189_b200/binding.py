@@ -51,7 +51,8 @@ EXPORTS = ["t5_create", "t5_destroy", "t5_last_error", "t5_param_count", "t5_par
            "t5_decode_begin", "t5_decode_step",
            "t5_launch_count", "t5_relpos_buckets", "t5_xent_zloss",
            "t5_gemm", "t5_attention", "t5_attention_backward_noalloc",
-           "t5_attention_ds_scratch_bytes", "t5_attention_backward_onepass"]
+           "t5_attention_ds_scratch_bytes", "t5_attention_backward_onepass",
+           "t5_kernel_status_word", "t5_selftest_bounded_wait"]
 
 _lib = None
 
@@ -89,6 +90,8 @@ def lib():
         L.t5_encode.argtypes = [vp, vp, C.POINTER(t5_batch), vp, vp, i64, vp]
         L.t5_decode_logits.argtypes = [vp, vp, C.POINTER(t5_batch), vp, vp, vp, i64, vp]
         L.t5_device_status.argtypes = [vp, vp, vp]
+        L.t5_kernel_status_word.argtypes = [vp]
+        L.t5_selftest_bounded_wait.argtypes = [vp, i64, vp]
         L.t5_profile_enable.argtypes = [vp, i32]
         L.t5_profile_read.argtypes = [vp, C.POINTER(C.c_double * 8), C.POINTER(C.c_double * 8),
                                       C.POINTER(i64 * 8)]
@@ -343,3 +346,15 @@ def t5_attention_backward_noalloc(impl, B, H, Tq, Tk, d_kv, causal, scale, q, k,
                                                _ptr(code_k), _ptr(bias_delta), _ptr(do), do.stride(0),
                                                _ptr(dq), dq.stride(0), _ptr(dk), dk.stride(0), _ptr(dv),
                                                dv.stride(0), _ptr(dbias_delta), _stream()))
+
+
+def t5_kernel_status_word(status):
+    """Hands the kernel-level entry points (t5_attention, ..., t5_gemm) a device int32 for their bounded waits
+    to report into; None switches reporting off."""
+    _check(lib().t5_kernel_status_word(_ptr(status)))
+
+
+def t5_selftest_bounded_wait(status, limit_cycles):
+    """One CTA waits, with the kernels' own bounded wait, on a barrier nothing arrives at; it gives up after
+    limit_cycles and leaves code 99 in `status` (device int32)."""
+    _check(lib().t5_selftest_bounded_wait(_ptr(status), int(limit_cycles), _stream()))

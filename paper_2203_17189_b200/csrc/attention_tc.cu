@@ -7,16 +7,24 @@
 //     dP = dO V^T,  dS = P (dP - delta_i),  dQ = scale dS K,  dK = scale dS^T Q,  dV = P^T dO,
 //     dbias_delta[h, j-i] += dS_ij.
 //
-// All three kernels use 128 threads (thread r owns tensor-memory lane r = one row of
-// the score tile), TMA loads into 128-byte-swizzled tiles, one elected thread issuing
-// the MMAs, and bounded mbarrier waits.  Several CTAs share an SM so that one CTA's
-// softmax overlaps another CTA's MMAs.
-//   forward : CTA = 128 queries x all keys (128-key tiles); online max/sum, output rows
-//             rescaled in registers.
-//   dQ      : CTA = 128 queries x all keys (64-key tiles); dQ accumulates in tensor memory;
-//             dS is also reduced along diagonals into the bias gradient.
-//   dK, dV  : CTA = 128 keys x all queries (64-query tiles), scores transposed (thread = key);
-//             dK and dV accumulate in tensor memory.
+// Every kernel loads its operands with TMA into 128-byte-swizzled tiles, keeps scores and accumulators in tensor
+// memory (thread r of a softmax warp group owns tensor-memory lane r = one row of the score tile), lets one
+// thread (or one elected lane) issue the MMAs, and bounds every mbarrier wait.  Several CTAs share an SM so that
+// one CTA's softmax overlaps another CTA's MMAs.
+//   attn_fwd_tc_kernel        128 threads, CTA = 128 queries x all keys in 64-key tiles; S and the output
+//                             accumulator in tensor memory, the accumulator rescaled in place and only when a row
+//                             maximum grew by more than 2^8; key tiles without a valid pair (packed rows) left out.
+//   backward, one pass over the scores (default whenever the caller provides the dS scratch: the training step
+//   and t5_attention_backward_onepass):
+//     attn_bwd_kvf_tc_kernel    320 threads (eight softmax warps, one MMA warp, one load / store warp), CTA = 128
+//                               keys x all queries in 64-query tiles: dK, dV, the bias gradient and a bf16 copy
+//                               of dS^T in the scratch [B*H, Tk^128, Tq^64].
+//     attn_bwd_dq_ds_tc_kernel  192 threads, CTA = 128 queries: dQ = scale dS K from the stored dS^T.
+//   backward, two kernels that each recompute the scores (t5_attention with backward = 1,
+//   t5_attention_backward_noalloc, configuration flag bit 17: no scratch needed):
+//     attn_bwd_dq_tc_kernel     256 threads, CTA = 128 queries x 64-key tiles; dQ in tensor memory; bias gradient.
+//     attn_bwd_dkv_tc_kernel    256 threads, CTA = 128 keys x 64-query tiles, transposed scores; dK, dV.
+//   attn_delta_tc_kernel      delta = rowsum(dO * O) from the float32 copy of O, ahead of either backward.
 #include "attention_tc.cuh"
 
 namespace {

@@ -154,6 +154,11 @@ cudaError_t attn_bwd_simt(int dtype, const AttnArgs& a, cudaStream_t st);
 bool attn_tc_supported(const AttnArgs& a);
 cudaError_t attn_fwd_tc(const AttnArgs& a, int* d_status, cudaStream_t st);
 cudaError_t attn_bwd_tc(const AttnArgs& a, int* d_status, cudaStream_t st);
+// status word the kernel-level entry points of the C ABI hand to the tcgen05 kernels (NULL: none)
+extern int32_t* g_kernel_status;
+// One CTA waits, with the kernels' own bounded wait, on a barrier nothing ever arrives at: after limit_cycles it
+// gives up, writes code 99 into *d_status and returns (exercises the give-up path without any hang)
+cudaError_t launch_selftest_bounded_wait(int* d_status, long long limit_cycles, cudaStream_t st);
 
 // element-wise / row kernels
 // dec_prefix (optional 0/1 flags): flagged positions get T5_PREFIX_BIT in their code and loss weight 0

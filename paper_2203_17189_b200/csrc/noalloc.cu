@@ -67,7 +67,7 @@ extern "C" int t5_attention_backward_noalloc(
     e = attn_bwd_simt(dtype, a, st);
   } else {
     if (dtype != DT_BF16 || !attn_tc_supported(a)) return T5_ERR_ARG;
-    e = attn_bwd_tc(a, nullptr, st);
+    e = attn_bwd_tc(a, g_kernel_status, st);
   }
   return e == cudaSuccess ? T5_OK : T5_ERR_CUDA;
 }

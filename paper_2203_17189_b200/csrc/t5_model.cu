@@ -961,6 +961,10 @@ int end_call(t5_handle* h, Ctx& cx) {
 }  // namespace
 
 // =============================================================================== C ABI
+// Status word of the kernel-level entry points below (t5_attention, t5_attention_backward_onepass, t5_gemm and the
+// allocation-free attention backward): they have no workspace whose first word could serve.  NULL: no reporting.
+int32_t* g_kernel_status = nullptr;
+
 extern "C" {
 
 int t5_create(const t5_config* cfg, t5_handle** out) {
@@ -1324,6 +1328,18 @@ int t5_xent_zloss(int32_t dtype, void* d_logits, const int32_t* d_targets, int32
   return e == cudaSuccess ? T5_OK : T5_ERR_CUDA;
 }
 
+int t5_kernel_status_word(int32_t* d_status) {
+  g_kernel_status = d_status;
+  return T5_OK;
+}
+
+int t5_selftest_bounded_wait(int32_t* d_status, int64_t limit_cycles, void* stream) {
+  if (!d_status) return T5_ERR_NULL;
+  if (limit_cycles < 1 || limit_cycles > 4000000000ll) return T5_ERR_ARG;
+  cudaError_t e = launch_selftest_bounded_wait(d_status, limit_cycles, (cudaStream_t)stream);
+  return e == cudaSuccess ? T5_OK : T5_ERR_CUDA;
+}
+
 int t5_attention(int32_t dtype, int32_t impl, int32_t backward, int32_t B, int32_t H, int32_t Tq, int32_t Tk,
                  int32_t d_kv, int32_t causal, float scale, const void* d_q, int32_t ldq, const void* d_k,
                  int32_t ldk, const void* d_v, int32_t ldv, void* d_o, int32_t ldo, float* d_o32, float* d_lse,
@@ -1348,7 +1364,7 @@ int t5_attention(int32_t dtype, int32_t impl, int32_t backward, int32_t B, int32
     e = backward ? attn_bwd_simt(dtype, a, st) : attn_fwd_simt(dtype, a, st);
   } else {
     if (dtype != DT_BF16 || !attn_tc_supported(a)) return T5_ERR_ARG;
-    e = backward ? attn_bwd_tc(a, nullptr, st) : attn_fwd_tc(a, nullptr, st);
+    e = backward ? attn_bwd_tc(a, g_kernel_status, st) : attn_fwd_tc(a, g_kernel_status, st);
   }
   return e == cudaSuccess ? T5_OK : T5_ERR_CUDA;
 }
@@ -1384,7 +1400,7 @@ int t5_attention_backward_onepass(int32_t B, int32_t H, int32_t Tq, int32_t Tk, 
   a.bias_far = bias_far; a.ds_scratch = d_ds_scratch; a.ds_bytes = ds_scratch_bytes;
   a.packed = 1;      // the codes may describe packed rows: keep the tile-skipping bookkeeping on
   if (!attn_tc_supported(a) || !attn_tc_onepass_supported(a)) return T5_ERR_ARG;
-  cudaError_t e = attn_bwd_tc(a, nullptr, (cudaStream_t)stream);
+  cudaError_t e = attn_bwd_tc(a, g_kernel_status, (cudaStream_t)stream);
   return e == cudaSuccess ? T5_OK : T5_ERR_CUDA;
 }
 
@@ -1403,7 +1419,7 @@ int t5_gemm(int32_t dtype, int32_t impl, int32_t M, int32_t N, int32_t K, float 
   } else {
     if (dtype != DT_BF16 || !gemm_tc_supported(g)) return T5_ERR_ARG;
     g.pair = impl == 2;
-    e = gemm_tc(g, nullptr, (cudaStream_t)stream);
+    e = gemm_tc(g, g_kernel_status, (cudaStream_t)stream);
   }
   return e == cudaSuccess ? T5_OK : T5_ERR_CUDA;
 }

@@ -33,20 +33,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false (and raises the CTA-wide abort flag) if the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          int code) {
+// Bounded wait.  Returns false (and raises the CTA-wide abort flag) if the limit ran out; the first wait of a
+// launch that gives up leaves its code in the status word.
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                                int code, long long limit_cycles) {
   if (mbar_try_wait(bar, parity)) return true;
   long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) {
+    if (clock64() - t0 > limit_cycles) {
       *abort_flag = 1;
       if (status) atomicCAS(status, 0, code);
       return false;
     }
   }
   return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          int code) {
+  return mbar_wait_limit(bar, parity, abort_flag, status, code, kWaitCycles);
 }
 
 // The same bounded wait for warps that share their SM's issue slots with busy arithmetic warps: between polls the

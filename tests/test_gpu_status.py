@@ -46,3 +46,28 @@ def test_step_clears_a_stale_status_word():
     torch.cuda.synchronize()
     h.t5_device_status(ws)
     assert torch.isfinite(loss4).all()
+
+
+def test_bounded_wait_gives_up_and_reports():
+    """The kernels' wait routine on a barrier nothing arrives at: it must give up after its limit, leave its code
+    in the status word and return normally (no trap, no hang); the context stays usable afterwards."""
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    Bd.t5_selftest_bounded_wait(status, 2_000_000)          # about a millisecond of SM cycles
+    torch.cuda.synchronize()
+    assert int(status.item()) == 99
+    with pytest.raises(Bd.T5Error):
+        Bd.t5_selftest_bounded_wait(status, 0)
+    # the device still works: a tensor-core GEMM through the kernel-level entry point, with a status word attached
+    status.zero_()
+    Bd.t5_kernel_status_word(status)
+    try:
+        a = torch.randn(256, 128, device=DEV).to(torch.bfloat16)
+        b = torch.randn(384, 128, device=DEV).to(torch.bfloat16)
+        d = torch.empty(256, 384, dtype=torch.bfloat16, device=DEV)
+        Bd.t5_gemm(1, 256, 384, 128, 1.0, a, 128, True, b, 128, True, d, 384)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        ref = a.float() @ b.float().T
+        assert (d.float() - ref).abs().max() <= 2e-2 * ref.abs().max()
+    finally:
+        Bd.t5_kernel_status_word(None)
