@@ -198,6 +198,28 @@ T5_API int t5_decode_step(t5_handle* h, const void* d_params, void* d_cache, int
                           int32_t Tmax, int32_t t, const int32_t* d_tokens, void* d_logits, void* d_workspace,
                           int64_t workspace_bytes, void* stream);
 
+/* Data-parallel training ("XLA GSPMD partitioning" section: data parallelism
+ * with replicated parameters; the partitioner there inserts the gradient
+ * all-reduce, here the caller does, overlapped with the backward pass).
+ * While t5_train_step_fwd_bwd enqueues its backward pass it calls the hook, on
+ * the calling host thread, each time a contiguous range of the gradient buffer
+ * has received its last write - the decoder's layers from the last to the
+ * first, then the encoder's, then the remaining tensors (embedding, bias
+ * tables, final norms, output head):
+ *   offset, count  element range of d_grads (float32) that is final;
+ *   d_rank_weight  device float: W_r, this call's number of loss-carrying
+ *                  target positions (the gradients are normalised by it);
+ *   stream         a CUDA stream on which everything that writes the range
+ *                  has been enqueued: work the hook enqueues behind an event
+ *                  recorded on it (e.g. scaling by W_r and an all-reduce on a
+ *                  communication stream) sees the final values while the rest
+ *                  of the backward pass keeps running.  The stream belongs to
+ *                  the library or the caller; the hook must not block on it.
+ * The ranges of one call are disjoint and cover the whole buffer.  fn = NULL
+ * removes the hook.  T5_ERR_NULL without a handle. */
+typedef void (*t5_grad_ready_fn)(void* user, int64_t offset, int64_t count, const float* d_rank_weight, void* stream);
+T5_API int t5_set_grad_hook(t5_handle* h, t5_grad_ready_fn fn, void* user);
+
 /* Reads back the status word the kernels of the last call on this workspace
  * left behind (their waits on TMA/tensor-core barriers are bounded; one that
  * runs out records a code instead of spinning).  SYNCHRONISES the stream.

@@ -44,6 +44,9 @@ class t5_profile_launch(C.Structure):
                 ("K", C.c_int32), ("ms", C.c_float)]
 
 
+# void hook(void* user, int64 offset, int64 count, const float* d_rank_weight, void* stream)
+GRAD_HOOK = C.CFUNCTYPE(None, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p)
+
 EXPORTS = ["t5_create", "t5_destroy", "t5_last_error", "t5_param_count", "t5_param_tensors",
            "t5_param_manifest", "t5_workspace_bytes", "t5_init_params", "t5_train_step_fwd_bwd",
            "t5_encode", "t5_decode_logits", "t5_device_status", "t5_profile_enable", "t5_profile_read",
@@ -52,7 +55,7 @@ EXPORTS = ["t5_create", "t5_destroy", "t5_last_error", "t5_param_count", "t5_par
            "t5_launch_count", "t5_relpos_buckets", "t5_xent_zloss",
            "t5_gemm", "t5_attention", "t5_attention_backward_noalloc",
            "t5_attention_ds_scratch_bytes", "t5_attention_backward_onepass",
-           "t5_kernel_status_word", "t5_selftest_bounded_wait"]
+           "t5_kernel_status_word", "t5_selftest_bounded_wait", "t5_set_grad_hook"]
 
 _lib = None
 
@@ -90,6 +93,7 @@ def lib():
         L.t5_encode.argtypes = [vp, vp, C.POINTER(t5_batch), vp, vp, i64, vp]
         L.t5_decode_logits.argtypes = [vp, vp, C.POINTER(t5_batch), vp, vp, vp, i64, vp]
         L.t5_device_status.argtypes = [vp, vp, vp]
+        L.t5_set_grad_hook.argtypes = [vp, GRAD_HOOK, vp]
         L.t5_kernel_status_word.argtypes = [vp]
         L.t5_selftest_bounded_wait.argtypes = [vp, i64, vp]
         L.t5_profile_enable.argtypes = [vp, i32]
@@ -279,6 +283,15 @@ class Handle:
         n = C.c_int64()
         _check(lib().t5_launch_count(self._h, C.byref(n)), self._h)
         return n.value
+
+    def t5_set_grad_hook(self, fn):
+        """fn(offset, count, rank_weight_ptr, stream_ptr) is called from inside t5_train_step_fwd_bwd as ranges of the
+        gradient buffer become final; None removes the hook.  The wrapper object is kept alive by the handle."""
+        if fn is None:
+            self._grad_hook = GRAD_HOOK()
+        else:
+            self._grad_hook = GRAD_HOOK(lambda user, off, cnt, w, st: fn(off, cnt, w, st))
+        _check(lib().t5_set_grad_hook(self._h, self._grad_hook, None), self._h)
 
     def t5_device_status(self, workspace):
         _check(lib().t5_device_status(self._h, _ptr(workspace), _stream()), self._h)

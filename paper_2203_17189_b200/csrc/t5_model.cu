@@ -86,6 +86,9 @@ struct t5_handle {
   size_t sync_next = 0;
   cudaEvent_t reader_events[8] = {};         // one per scratch buffer the side stream reads
   std::vector<cudaEvent_t> layer_events;     // per decoder layer: its cross-attention keys / values are projected
+  // data-parallel training: called as ranges of the gradient buffer become final (see t5_set_grad_hook)
+  t5_grad_ready_fn grad_hook = nullptr;
+  void* grad_hook_user = nullptr;
 };
 
 namespace {
@@ -786,6 +789,19 @@ void decoder_forward(Ctx& cx, const void* enc_src, RowNorm enc_rn, void* logits_
            row_norm(cx, w.dec_ssq_f), "logits");
 }
 
+// Elements [begin, end) of the gradient buffer are final once the work enqueued so far is done: tell the caller's
+// hook, with a stream that follows all of that work (the side stream, made to wait for the main stream first, when
+// the weight-gradient GEMMs run there; else the caller's own stream).
+void grads_ready(Ctx& cx, int64_t begin, int64_t end) {
+  if (!cx.h->grad_hook || cx.err != cudaSuccess || end <= begin) return;
+  cudaStream_t s = cx.st;
+  if (cx.side) {
+    fork_to_side(cx);
+    s = cx.side;
+  }
+  if (cx.err == cudaSuccess) cx.h->grad_hook(cx.h->grad_hook_user, begin, end - begin, cx.w->W_f, (void*)s);
+}
+
 void backward(Ctx& cx, const t5_batch* b) {
   Workspace& w = *cx.w;
   const t5_config& c = cx.h->cfg;
@@ -816,6 +832,7 @@ void backward(Ctx& cx, const t5_batch* b) {
       first_cross = false;
     }
     attn_backward(cx, cx.h->dec[l].self, w.dec_self[l], w.dX_dec, w.dXb_dec, gs, nullptr, kNoNorm, nullptr, 0);
+    grads_ready(cx, cx.h->dec[l].self.norm, l + 1 < c.n_dec_layers ? cx.h->dec[l + 1].self.norm : cx.h->dec_final_norm);
   }
   wait_readers(cx, BUF_EMBED_GRAD);      // the embedding gradient must hold the logits' share before rows are added to it
   CKL(CAT_EMBED, 1, launch_embed_scatter_add(w.dec_in, w.dX_dec, cx.grads + cx.h->token_embed, (int)Nd, d, cx.st),
@@ -823,7 +840,11 @@ void backward(Ctx& cx, const t5_batch* b) {
   CKL(CAT_MISC, 1, launch_relbias_fold(cx.h->spec_dec, w.dbias_dec, H, cx.Td, cx.Td, c.rel_buckets, cx.grads + cx.h->dec_relbias,
                          cx.st),
      "relbias fold dec");
-  if (!encdec) return;
+  if (!encdec) {
+    grads_ready(cx, 0, cx.h->dec[0].self.norm);                       // embedding, bias table
+    grads_ready(cx, cx.h->dec_final_norm, cx.h->n_params);            // final norm, separate output head
+    return;
+  }
   wait_readers(cx, BUF_DY32);      // the encoder-output gradient is complete
   norm_backward(cx, cx.h->enc_final_norm, w.enc_x_final, w.enc_ssq_f, w.dY32, 1, nullptr, w.dX_enc, w.dXb_enc, (int)Ne,
                 "enc final norm bwd");
@@ -831,12 +852,16 @@ void backward(Ctx& cx, const t5_batch* b) {
   for (int l = c.n_enc_layers - 1; l >= 0; --l) {
     ffn_backward(cx, cx.h->enc[l].ffn, w.enc_ffn[l], w.dX_enc, w.dXb_enc, Ne);
     attn_backward(cx, cx.h->enc[l].attn, w.enc_attn[l], w.dX_enc, w.dXb_enc, ge, nullptr, kNoNorm, nullptr, 0);
+    grads_ready(cx, cx.h->enc[l].attn.norm, l + 1 < c.n_enc_layers ? cx.h->enc[l + 1].attn.norm : cx.h->enc_final_norm);
   }
   CKL(CAT_EMBED, 1, launch_embed_scatter_add(b->d_enc_tokens, w.dX_enc, cx.grads + cx.h->token_embed, (int)Ne, d, cx.st),
      "embed scatter enc");
   CKL(CAT_MISC, 1, launch_relbias_fold(cx.h->spec_enc, w.dbias_enc, H, cx.Te, cx.Te, c.rel_buckets, cx.grads + cx.h->enc_relbias,
                          cx.st),
      "relbias fold enc");
+  grads_ready(cx, cx.h->dec_final_norm, cx.h->n_params);              // decoder final norm, separate output head
+  grads_ready(cx, cx.h->enc_final_norm, cx.h->dec[0].self.norm);      // encoder final norm, decoder bias table
+  grads_ready(cx, 0, cx.h->enc[0].attn.norm);                         // embedding, encoder bias table
 }
 
 // ---- incremental decoding: the caller's cache buffer holds, per decoder layer, the self-attention keys / values of the
@@ -1088,6 +1113,13 @@ int t5_adamw_update(t5_handle* h, void* d_params, float* d_master, float* d_m, f
     i = j + 1;
   }
   if (e != cudaSuccess) return fail(h, T5_ERR_CUDA, "adamw: %s", cudaGetErrorString(e));
+  return T5_OK;
+}
+
+int t5_set_grad_hook(t5_handle* h, t5_grad_ready_fn fn, void* user) {
+  if (!h) return T5_ERR_NULL;
+  h->grad_hook = fn;
+  h->grad_hook_user = user;
   return T5_OK;
 }
 

@@ -50,3 +50,76 @@ def combine(grads: torch.Tensor, loss4: torch.Tensor, group=None, bucket_element
     loss4[:3] = parts
     loss4[3:4] = w_total
     return float(w_total.item())
+
+
+class _DeviceFloat:
+    """A float32 scalar at a raw device address, for torch.as_tensor (CUDA array interface)."""
+
+    def __init__(self, ptr):
+        self.__cuda_array_interface__ = {"shape": (1,), "typestr": "<f4", "data": (int(ptr), False), "version": 2}
+
+
+class OverlappedReducer:
+    """Gradient all-reduce that runs while the backward pass is still going.
+
+    The library reports each range of the gradient buffer as soon as its last write is enqueued (t5_set_grad_hook).
+    For every range this class multiplies the rank's values by W_r (the rank's target count, read on the device), and
+    starts a sum all-reduce on a communication stream behind an event recorded on the stream the library names;
+    nothing blocks the host or the compute streams.  finish() then waits for the collectives, all-reduces W and the
+    loss parts, and divides by the job's W:  grads <- sum_r W_r g_r / W,  loss4 <- [L, ce, z-part, W] of the job -
+    the same result as combine().  reduce_range() is the hook body and can be driven by hand (CPU tensors, gloo)."""
+
+    def __init__(self, grads: torch.Tensor, group=None):
+        self.grads, self.group = grads, group
+        self.comm = torch.cuda.Stream(device=grads.device) if grads.is_cuda else None
+        self.pending, self.ranges = [], []
+
+    def attach(self, handle):
+        handle.t5_set_grad_hook(self._hook)
+        return self
+
+    def _hook(self, offset, count, weight_ptr, stream_ptr):
+        w = torch.as_tensor(_DeviceFloat(weight_ptr), device=self.grads.device)
+        self.reduce_range(offset, count, w, stream_ptr)
+
+    def reduce_range(self, offset, count, rank_weight, stream_ptr=None):
+        """rank_weight: one-element float32 tensor on the gradients' device holding W_r."""
+        self.ranges.append((int(offset), int(count)))
+        view = self.grads[offset:offset + count]
+        active = dist.is_initialized() and dist.get_world_size(self.group) > 1
+        if self.comm is None:
+            view.mul_(rank_weight)
+            if active:
+                self.pending.append(dist.all_reduce(view, op=dist.ReduceOp.SUM, group=self.group, async_op=True))
+            return
+        ready = torch.cuda.Event()
+        if stream_ptr:
+            ready.record(torch.cuda.ExternalStream(int(stream_ptr), device=self.grads.device))
+        else:       # a null handle is the default stream
+            ready.record(torch.cuda.default_stream(self.grads.device))
+        self.comm.wait_event(ready)
+        with torch.cuda.stream(self.comm):
+            view.mul_(rank_weight)
+            if active:
+                self.pending.append(dist.all_reduce(view, op=dist.ReduceOp.SUM, group=self.group, async_op=True))
+
+    def finish(self, loss4: torch.Tensor):
+        """Call after t5_train_step_fwd_bwd returned (on the stream it was given).  Returns the job's W."""
+        for work in self.pending:
+            work.wait()
+        self.pending = []
+        if self.comm is not None:
+            torch.cuda.current_stream(self.grads.device).wait_stream(self.comm)
+        active = dist.is_initialized() and dist.get_world_size(self.group) > 1
+        w_total = loss4[3:4].clone()
+        parts = loss4[:3] * loss4[3:4]
+        if active:
+            dist.all_reduce(w_total, op=dist.ReduceOp.SUM, group=self.group)
+            dist.all_reduce(parts, op=dist.ReduceOp.SUM, group=self.group)
+        inv = torch.where(w_total > 0, 1.0 / torch.clamp(w_total, min=1.0), torch.zeros_like(w_total))
+        self.grads.mul_(inv.to(self.grads.dtype))
+        loss4[:3] = parts * inv
+        loss4[3:4] = w_total
+        covered = sorted(self.ranges)
+        self.ranges = []
+        return float(w_total.item()), covered
