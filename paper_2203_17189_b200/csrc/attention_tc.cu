@@ -198,6 +198,10 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
     const int tcode = tile_code64(codes_s + k0, tid & 31);
     const bool fast = tcode > 0 && __all_sync(0xffffffffu, cq == tcode) &&
                       (!p.causal || k0 + 63 <= q0 + (warp << 5));          // warp-uniform: no mask needed
+    // All keys of the tile carry one code and none lies ahead of a row of this warp: a row then sees the whole tile
+    // or nothing of it (padding rows, rows of another segment), so no entry needs a test of its own
+    const bool by_row = !fast && tcode > 0 && (!p.causal || k0 + 63 <= q0 + (warp << 5));
+    const bool row_ok = !by_row || ((cq ^ tcode) & ~T5_PREFIX_BIT) == 0;
     const float* brow = bias_s + (k0 - tid + 127);
     // the whole tile lies where the bias no longer depends on the distance (saturated bucket): one value, no loads
     const bool flat = has_bias && p.bias_far > 0 && (k0 - (q0 + 127) >= p.bias_far || q0 - (k0 + 63) >= p.bias_far);
@@ -220,7 +224,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
 #pragma unroll
           for (int jj = 0; jj < 32; ++jj) sc[c][jj] = __uint_as_float(r[c][jj]) * sc2;
         }
-        if (!fast) {
+        if (!fast && !by_row) {
 #pragma unroll
           for (int jj = 0; jj < 32; ++jj) {
             int j = k0 + c * 32 + jj;
@@ -244,11 +248,13 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
     // probabilities hold as well as values below one, and the accumulator rows need no rescaling.  The result
     // O = acc / l and lse = m_run + log2(l) do not depend on which reference point was used.
     constexpr float kLazy = 8.f;
-    const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+    // a row that sees nothing of the tile (see by_row): no maximum, and below every probability becomes 2^-inf = 0
+    const float m_tile = row_ok ? fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) : -INFINITY;
     const bool grow = m_tile > m_run + kLazy || (m_run == -INFINITY && m_tile != -INFINITY);
     const bool warp_moves = __any_sync(0xffffffffu, grow);
     const float m_new = warp_moves ? fmaxf(m_run, m_tile) : m_run;      // a warp that rescales moves all its rows
     const float m_eff = m_new == -INFINITY ? 0.f : m_new;      // a row with no valid key so far: exp2(-inf - 0) = 0
+    const float m_exp = row_ok ? m_eff : INFINITY;
     const float corr = ex2_approx(m_run - m_eff);
     // rescale the accumulator rows of this warp if any of their reference points moved
     if (u > 0 && warp_moves) {
@@ -271,7 +277,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant
         uint32_t u[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          u[e] = pack_bf16(ex2_approx(sc[c][q8 * 8 + 2 * e] - m_eff), ex2_approx(sc[c][q8 * 8 + 2 * e + 1] - m_eff));
+          u[e] = pack_bf16(ex2_approx(sc[c][q8 * 8 + 2 * e] - m_exp), ex2_approx(sc[c][q8 * 8 + 2 * e + 1] - m_exp));
           // the row sum uses the bf16-rounded probabilities, so the weights the MMA applies sum to one
           ls[e] += bf16_lo(u[e]) + bf16_hi(u[e]);
         }
@@ -947,6 +953,7 @@ struct KvfBars {
   uint64_t qd_full[2], qd_free[2];
   uint64_t s_full, s_free, p_full, p_free;
   uint64_t acc;
+  uint64_t list;       // packed rows: the list of query tiles is in shared memory
   uint32_t tmem;
   int abort_flag;
 };
@@ -1003,28 +1010,35 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
     mbar_init(&bars->p_full, 8);         // one arrival per softmax warp
     mbar_init(&bars->p_free, 2);         // the accumulating MMAs are done + the dS store has read the tile
     mbar_init(&bars->acc, 1);
+    mbar_init(&bars->list, 1);
     bars->abort_flag = 0;
     fence_barrier_init();
   }
-  auto first_loads = [&]() {
-    if (n > 0) {
+  // The loading warp, ahead of the CTA-wide barrier: K and V go out at once; on packed rows it then makes the list of
+  // query tiles (those whose 128-query block shares a segment with this CTA's keys: the dQ kernel applies the same
+  // rule, so the regions of the dS scratch that stay unwritten are never read), sends the first Q / dO tiles and
+  // publishes the list; the other warps pick it up when they need it.
+  const bool kv_loaded = n > 0;
+  if (warp == 9) {
+    if (lane == 0 && kv_loaded) {
       mbar_arrive_expect_tx(&bars->kv, 2 * L::kKVBytes);
 #pragma unroll
       for (int c = 0; c < DK / 64; ++c) {
         tma_load_3d(smem + L::kK + c * 16384, &mk, h * DK + c * 64, k0, b, &bars->kv);
         tma_load_3d(smem + L::kV + c * 16384, &mv, h * DK + c * 64, k0, b, &bars->kv);
       }
-      for (int i = 0; i < NST && i < n; ++i) load_qd(i);
     }
-  };
-  if (!p.packed) {
-    if (tid == 9 * 32) first_loads();
-  } else {
-    // packed rows: query tiles whose 128-query block shares no segment with this CTA's keys are left out (the dQ
-    // kernel applies the same rule, so the regions of the dS scratch that stay unwritten are never read)
-    n = packed_tile_list<kKvfThreads>(p.code_k + (int64_t)b * p.Tk, p.Tk, k0, p.code_q + (int64_t)b * p.Tq, p.Tq, t_begin,
-                                      n_qt, qt_s, tid);
-    if (tid == 9 * 32) first_loads();
+    __syncwarp();
+    if (p.packed) {
+      n = packed_tile_list_warp(p.code_k + (int64_t)b * p.Tk, p.Tk, k0, p.code_q + (int64_t)b * p.Tq, p.Tq, t_begin, n_qt,
+                                qt_s, lane);
+      if (lane == 0) qt_s[n_qt] = n;
+      __syncwarp();
+    }
+    if (lane == 0) {
+      for (int i = 0; i < NST && i < n; ++i) load_qd(i);
+      if (p.packed) mbar_arrive(&bars->list);
+    }
   }
   if (warp == 8) tmem_alloc(&bars->tmem, kTmemCols);
   const int span = p.Tq + p.Tk - 1;
@@ -1033,9 +1047,15 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem;
   bool ok = true;
+  if (p.packed && warp == 8) {
+    ok = __all_sync(0xffffffffu, mbar_wait_relaxed(&bars->list, 0, abort_flag, p.status, 39));
+    n = ok ? qt_s[n_qt] : 0;
+  }
 
   if (warp == 9) {
     // ------------------------------------------------------------------ loads and the dS store
+    if (lane == 0 && n == 0 && kv_loaded)      // every tile was left out: K and V must still land before the CTA ends
+      mbar_wait_relaxed(&bars->kv, 0, abort_flag, p.status, 38);
     if (lane == 0 && n > 0) {
       for (int i = 0; i < n && ok; ++i) {
         ok = mbar_wait_relaxed(&bars->p_full, i & 1, abort_flag, p.status, 41);
@@ -1143,6 +1163,10 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
       if (want_db)
         for (int w = tid; w < nb; w += kKvfSoftmaxThreads) dbias_s[w] = 0.f;
       asm volatile("bar.sync 1, 256;" ::: "memory");
+    }
+    if (p.packed) {
+      ok = __all_sync(0xffffffffu, mbar_wait_relaxed(&bars->list, 0, abort_flag, p.status, 40));
+      n = ok ? qt_s[n_qt] : 0;
     }
     const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
     const float sc2 = p.scale * kLog2e;
@@ -1380,7 +1404,8 @@ attn_bwd_dq_ds_tc_kernel(const __grid_constant__ CUtensorMap mds, const __grid_c
   uint64_t* full = (uint64_t*)(smem + L::kBar);
   uint64_t* empty = full + NST;
   uint64_t* done = empty + NST;
-  uint32_t* tmem_holder = (uint32_t*)(done + 1);
+  uint64_t* list_bar = done + 1;      // packed rows: the list of key tiles is in shared memory
+  uint32_t* tmem_holder = (uint32_t*)(list_bar + 1);
   volatile int* abort_flag = (volatile int*)(tmem_holder + 1);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * 128;
@@ -1393,18 +1418,30 @@ attn_bwd_dq_ds_tc_kernel(const __grid_constant__ CUtensorMap mds, const __grid_c
   if (tid == 0) {
     for (int s = 0; s < NST; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(done, 1);
+    mbar_init(list_bar, 1);
     *abort_flag = 0;
     fence_barrier_init();
   }
-  // packed rows: the key tiles the dK / dV kernel left out for these queries hold nothing it stored
-  if (p.packed)
-    n_kt = packed_tile_list<192>(p.code_q + (int64_t)b * p.Tq, p.Tq, q0, p.code_k + (int64_t)b * p.Tk, p.Tk, 0, n_kt, kt_s, tid);
+  // packed rows: the key tiles the dK / dV kernel left out for these queries hold nothing it stored.  The loading
+  // warp makes the list while the rest of the set-up runs and publishes it; the others pick it up behind the barrier.
+  const int t_end = n_kt;
+  if (p.packed && warp == 0) {
+    __syncwarp();
+    n_kt = packed_tile_list_warp(p.code_q + (int64_t)b * p.Tq, p.Tq, q0, p.code_k + (int64_t)b * p.Tk, p.Tk, 0, t_end, kt_s, lane);
+    if (lane == 0) kt_s[t_end] = n_kt;
+    __syncwarp();
+    if (lane == 0) mbar_arrive(list_bar);
+  }
   if (warp == 1) tmem_alloc(tmem_holder, kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
   bool ok = true;
+  if (p.packed && warp != 0) {
+    ok = __all_sync(0xffffffffu, mbar_wait(list_bar, 0, abort_flag, p.status, 54));
+    n_kt = ok ? kt_s[t_end] : 0;
+  }
 
   if (warp == 0) {
     if (lane == 0) {

@@ -92,51 +92,55 @@ struct Bars {
 // own rows holds none; its two tiles are left out.  The rule is taken per pair of 128-row blocks so that the kernel
 // that walks key blocks and the kernel that walks query blocks leave out exactly the same (query, key) regions (the
 // second one reads what the first one stored).
-// Writes the kept tiles of [t_begin, t_end) (t_begin even) in increasing order to list_s and returns their number.
-// list_s: shared memory, t_end + 2 ints.  Every thread of the CTA (NT of them) must call; contains barriers.
-template <int NT>
-__device__ int packed_tile_list(const int* own_codes, int T_own, int own0, const int* other_codes, int T_other,
-                                int t_begin, int t_end, int* list_s, int tid) {
-  const int warp = tid >> 5, lane = tid & 31;
-  int* own_rng = list_s + t_end;
-  auto range128 = [&](const int* codes, int T, int r0, int& lo, int& hi) {
-    lo = 0x7fffffff; hi = 0;
+// Writes the kept tiles of [t_begin, t_end) (t_begin even) in increasing order to list_s (shared memory, t_end ints)
+// and returns their number in every lane.  Run by ONE warp (all 32 lanes): every global load of the codes is
+// independent of the others, so the whole list costs about one round trip to L2; the caller publishes the list to
+// the other warps (an mbarrier arrive after __syncwarp).
+__device__ __forceinline__ int packed_tile_list_warp(const int* own_codes, int T_own, int own0, const int* other_codes,
+                                                     int T_other, int t_begin, int t_end, int* list_s, int lane) {
+  auto load4 = [&](const int* codes, int T, int r0, int (&c)[4]) {
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const int r = r0 + lane + 32 * k;
-      const int c = r < T ? (codes[r] & ~T5_PREFIX_BIT) : 0;
-      if (c) { lo = min(lo, c); hi = ::max(hi, c); }
+      c[k] = r < T ? (codes[r] & ~T5_PREFIX_BIT) : 0;
     }
+  };
+  auto range = [&](const int (&c)[4], int& lo, int& hi) {
+    lo = 0x7fffffff; hi = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (c[k]) { lo = min(lo, c[k]); hi = ::max(hi, c[k]); }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
       hi = ::max(hi, __shfl_xor_sync(0xffffffffu, hi, o));
     }
   };
-  int lo, hi;
-  if (warp == 0) {
-    range128(own_codes, T_own, own0, lo, hi);
-    if (lane == 0) { own_rng[0] = lo; own_rng[1] = hi; }
-  }
-  __syncthreads();
-  const int slo = own_rng[0], shi = own_rng[1];
-  for (int pb = t_begin / 2 + warp; 2 * pb < t_end; pb += NT / 32) {
-    range128(other_codes, T_other, pb * 128, lo, hi);
-    const int act = (shi > 0 && hi > 0 && hi >= slo && lo <= shi) ? 1 : 0;
-    if (lane == 0) {
-      list_s[2 * pb] = act;
-      if (2 * pb + 1 < t_end) list_s[2 * pb + 1] = act;
+  int own[4], slo, shi;
+  load4(own_codes, T_own, own0, own);
+  int n = 0;
+  // four 128-row blocks of the other side per round: sixteen loads per lane in flight
+  for (int pb0 = t_begin / 2; 2 * pb0 < t_end; pb0 += 4) {
+    int c[4][4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) load4(other_codes, T_other, (pb0 + q) * 128, c[q]);
+    if (pb0 == t_begin / 2) range(own, slo, shi);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      int lo, hi;
+      range(c[q], lo, hi);
+      const bool act = shi > 0 && hi > 0 && hi >= slo && lo <= shi;
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int t = 2 * (pb0 + q) + e;
+        if (act && t < t_end) {
+          if (lane == 0) list_s[n] = t;
+          ++n;
+        }
+      }
     }
   }
-  __syncthreads();
-  if (tid == 0) {      // compaction in place: the write position never passes the read position
-    int n = 0;
-    for (int t = t_begin; t < t_end; ++t)
-      if (list_s[t]) list_s[n++] = t;
-    own_rng[0] = n;
-  }
-  __syncthreads();
-  return own_rng[0];
+  return n;
 }
 
 // ----------------------------------------------------------------------------- host side
