@@ -1182,7 +1182,7 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
       ok = __all_sync(0xffffffffu, mbar_wait_relaxed(&bars->s_full, par, abort_flag, p.status, 46));
       if (!ok) break;
       tc_fence_after();
-#pragma unroll
+#pragma unroll 1
       for (int c = 0; c < 2; ++c) {
         const int cc = half * 32 + c * 16;                 // first of this pass's 16 queries within the tile
         const int qq0 = qb + cc;
