@@ -768,6 +768,12 @@ cudaError_t launch(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap& 
       (g_num_sms - rem) * 8 > g_num_sms * (tiles / g_num_sms + 1)) {
     grid = g_num_sms;
     p.sk_full = tiles / g_num_sms; p.sk_rem = rem; p.sk_flags = g.sk_flags;
+  } else if (g.sk_flags && g.out_f32 && !g.xg_out && k_blocks >= 32 && tiles * 2 <= g_num_sms && tiles <= 160 &&
+             (long long)k_blocks * tiles >= 4ll * g_num_sms) {
+    // fewer tiles than half the SMs and a long contraction (weight gradients of narrow layers): every tile is cut
+    // along K over all SMs - the same segments and flags as the tail above, with no full wave before them
+    grid = g_num_sms;
+    p.sk_full = 0; p.sk_rem = tiles; p.sk_flags = g.sk_flags;
   }
   kern<<<grid, kThreads, S::kTotal, st>>>(ma, mb, p);
   return cudaGetLastError();
@@ -795,6 +801,10 @@ cudaError_t launch2(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap&
   if (g.epi == 0 && g.sk_flags && g.out_f32 && !g.xg_out && rem > 0 && k_blocks >= 128 && tiles >= pairs && pairs <= 160 &&
       (pairs - rem) * 8 > pairs * (tiles / pairs + 1)) {
     p.sk_full = tiles / pairs; p.sk_rem = rem; p.sk_flags = g.sk_flags;
+  } else if (g.epi == 0 && g.sk_flags && g.out_f32 && !g.xg_out && k_blocks >= 32 && tiles * 2 <= pairs && tiles <= 160 &&
+             (long long)k_blocks * tiles >= 4ll * pairs) {
+    // fewer tiles than half the pairs and a long contraction: every tile is cut along K over all pairs
+    p.sk_full = 0; p.sk_rem = tiles; p.sk_flags = g.sk_flags;
   } else if (tiles < pairs) {
     pairs = tiles;
   }

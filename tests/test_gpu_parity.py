@@ -452,11 +452,13 @@ def test_gemm_tcgen05_strided_views():
 
 @pytest.mark.parametrize("impl", [1, 2])
 @pytest.mark.parametrize("ak,bk", [(0, 0), (1, 1)])
-@pytest.mark.parametrize("M,N,K", [(2048, 5120, 8192), (6144, 2048, 8192), (2048, 2048, 4096), (1000, 520, 1104)])
+@pytest.mark.parametrize("M,N,K", [(2048, 5120, 8192), (6144, 2048, 8192), (2048, 2048, 4096), (1000, 520, 1104),
+                                   (512, 384, 32768), (768, 768, 16384), (1152, 512, 8200), (296, 200, 9000)])
 def test_gemm_tcgen05_stream_k_tail(impl, ak, bk, M, N, K):
     """float32-output GEMMs whose last wave is partial: with long K its tiles are cut along K over all SMs
     (one segment stores, the others add atomically); result must equal the plain product.  The first two
-    shapes take that path in both kernels (single CTAs and CTA pairs), the others must not be disturbed."""
+    shapes take that path in both kernels (single CTAs and CTA pairs), the next two must not be disturbed; the
+    last four have far fewer tiles than SMs and a long K: every tile is cut along K over the whole GPU."""
     rng = np.random.default_rng(M + N + K)
     A = torch.from_numpy(rng.standard_normal((M, K)).astype(np.float32)).to(DEV).to(torch.bfloat16)
     Bm = torch.from_numpy(rng.standard_normal((N, K)).astype(np.float32)).to(DEV).to(torch.bfloat16)
