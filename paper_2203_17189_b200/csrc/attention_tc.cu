@@ -51,6 +51,7 @@ template <int DK>
 __global__ void __launch_bounds__(128)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
                    const __grid_constant__ CUtensorMap mv, TcParams p) {
+  pdl_sync();
   using L = FwdLayout<DK>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -882,6 +883,7 @@ template <int DK>
 __global__ void __launch_bounds__(256)
 attn_delta_tc_kernel(const bf16* __restrict__ O, int ldo, const float* __restrict__ O32, int ldo32,
                      const bf16* __restrict__ dO, int lddo, float* __restrict__ delta, int B, int H, int Tq) {
+  pdl_sync();
   const int per_row = H * DK / 8;
   const int64_t gt = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t n_rows = (int64_t)B * Tq;
@@ -968,6 +970,7 @@ attn_bwd_kvf_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_cons
                        const __grid_constant__ CUtensorMap mk, const __grid_constant__ CUtensorMap mv,
                        const __grid_constant__ CUtensorMap mds, const __grid_constant__ CUtensorMap mdk_out,
                        const __grid_constant__ CUtensorMap mdv_out, TcParams p) {
+  pdl_sync();
   using L = KvfLayout<DK>;
   constexpr int NST = L::kStages;
   extern __shared__ unsigned char smem_raw[];
@@ -1397,6 +1400,7 @@ struct DqsLayout {
 template <int DK>
 __global__ void __launch_bounds__(192)
 attn_bwd_dq_ds_tc_kernel(const __grid_constant__ CUtensorMap mds, const __grid_constant__ CUtensorMap mk, TcParams p) {
+  pdl_sync();
   using L = DqsLayout<DK>;
   constexpr int NST = L::kStages;
   extern __shared__ unsigned char smem_raw[];
@@ -1532,8 +1536,7 @@ cudaError_t fwd_launch(const AttnArgs& a, int* status, cudaStream_t st) {
   TcParams p = base_params(a, status);
   p.out0 = a.O; p.ld0 = a.ldo; p.o32 = a.O32; p.ldo32 = a.ldo32;
   dim3 grid((a.Tq + 127) / 128, a.H, a.B);
-  attn_fwd_tc_kernel<DK><<<grid, 128, smem, st>>>(mq, mk, mv, p);
-  return cudaGetLastError();
+  return launch_pdl(attn_fwd_tc_kernel<DK>, grid, dim3(128), smem, st, mq, mk, mv, p);
 }
 
 // One pass over the scores: kernel A (dK, dV, dS^T to scratch) then kernel B (dQ from the stored dS^T).
@@ -1555,8 +1558,7 @@ cudaError_t bwd_fused_launch(const AttnArgs& a, int* status, cudaStream_t st) {
     cudaError_t e = cudaFuncSetAttribute(attn_bwd_kvf_tc_kernel<DK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     dim3 grid((a.Tk + 127) / 128, a.H, a.B);
-    attn_bwd_kvf_tc_kernel<DK><<<grid, kKvfThreads, smem, st>>>(mq, mdo, mk, mv, mds_st, mdk_out, mdv_out, p);
-    e = cudaGetLastError();
+    e = launch_pdl(attn_bwd_kvf_tc_kernel<DK>, grid, dim3(kKvfThreads), smem, st, mq, mdo, mk, mv, mds_st, mdk_out, mdv_out, p);
     if (e != cudaSuccess) return e;
   }
   {
@@ -1565,8 +1567,7 @@ cudaError_t bwd_fused_launch(const AttnArgs& a, int* status, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     p.out0 = a.dQ; p.ld0 = a.lddq;
     dim3 grid((a.Tq + 127) / 128, a.H, a.B);
-    attn_bwd_dq_ds_tc_kernel<DK><<<grid, 192, smem, st>>>(mds_ld, mk64, p);
-    return cudaGetLastError();
+    return launch_pdl(attn_bwd_dq_ds_tc_kernel<DK>, grid, dim3(192), smem, st, mds_ld, mk64, p);
   }
 }
 
@@ -1574,9 +1575,9 @@ template <int DK>
 cudaError_t bwd_launch(const AttnArgs& a, int* status, cudaStream_t st) {
   int I = a.H * DK;
   const int64_t dthreads = (int64_t)a.B * a.Tq * (I / 8);
-  attn_delta_tc_kernel<DK><<<(unsigned)((dthreads + 255) / 256), 256, 0, st>>>(
-      (const bf16*)a.O, a.ldo, a.O32, a.ldo32, (const bf16*)a.dO, a.lddo, a.delta, a.B, a.H, a.Tq);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = launch_pdl(attn_delta_tc_kernel<DK>, dim3((unsigned)((dthreads + 255) / 256)), dim3(256), 0, st,
+                             (const bf16*)a.O, a.ldo, (const float*)a.O32, a.ldo32, (const bf16*)a.dO, a.lddo, a.delta, a.B, a.H,
+                             a.Tq);
   if (e != cudaSuccess) return e;
   if (attn_tc_onepass_supported(a)) return bwd_fused_launch<DK>(a, status, st);
   TcParams p = base_params(a, status);

@@ -73,6 +73,28 @@ __device__ __forceinline__ float rn_factor(const RowNorm& r, int64_t row) {
 }
 
 // ---------------------------------------------------------------------------
+// Programmatic dependent launch.  A kernel launched with launch_pdl may have its CTAs brought onto the SMs while the
+// kernel before it in the stream is still draining; pdl_sync(), the first thing such a kernel executes, holds every
+// thread until that earlier grid has completed and its writes are visible, and at once lets the kernel after this
+// one start its own launch.  What overlaps is launch latency and CTA set-up, never any access to global memory.
+// Under an ordinary launch both instructions do nothing.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_sync() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
+// ---------------------------------------------------------------------------
 // Launchers.  `dtype` selects float / bf16 storage for "T" tensors; all
 // reductions and accumulators are float32.  Every launcher returns the
 // cudaError_t of its launch.

@@ -245,6 +245,7 @@ __global__ void __launch_bounds__(256, 2)
 rmsnorm_bwd_rows_kernel(const TDY* __restrict__ dY, const float* __restrict__ X, RowNorm rn,
                         const T* __restrict__ g, const float* dX_in, float* dX_out, T* __restrict__ dXb,
                         float* __restrict__ partial, int rows, int d) {
+  pdl_sync();
   __shared__ float red[2][8];
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
   float4 gv[NCH], acc[NCH];
@@ -316,6 +317,7 @@ rmsnorm_bwd_rows_kernel(const TDY* __restrict__ dY, const float* __restrict__ X,
 }
 
 __global__ void colsum_kernel(const float* __restrict__ partial, int n_part, int d, float* __restrict__ out) {
+  pdl_sync();
   // block (32, 16): 32 columns, the partial rows split over 16 groups, then a shared-memory tree
   __shared__ float red[16][33];
   int c = blockIdx.x * 32 + threadIdx.x;
@@ -700,8 +702,8 @@ cudaError_t launch_rmsnorm_bwd(int dtype, const void* dy, int dy_f32, const floa
   if (d > 1024 && parts > 296) parts = 296;
   if (d <= 4096) {
 #define RBR(T, TDY, NCH)                                                                                          \
-  rmsnorm_bwd_rows_kernel<T, TDY, NCH><<<parts, 256, 0, st>>>((const TDY*)dy, X, rn, (const T*)g, dX_in, dX_out, \
-                                                              (T*)dXb, partial, rows, d)
+  launch_pdl(rmsnorm_bwd_rows_kernel<T, TDY, NCH>, dim3(parts), dim3(256), 0, st, (const TDY*)dy, X, rn, (const T*)g, \
+             dX_in, dX_out, (T*)dXb, partial, rows, d)
 #define RBR_N(T, TDY)                                                     \
   do {                                                                    \
     if (d <= 1024) RBR(T, TDY, 1); else if (d <= 2048) RBR(T, TDY, 2);    \
@@ -733,8 +735,7 @@ cudaError_t launch_rmsnorm_bwd(int dtype, const void* dy, int dy_f32, const floa
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  colsum_kernel<<<blocks_for(d, 32), dim3(32, 16), 0, st>>>(partial, parts, d, dg);
-  return cudaGetLastError();
+  return launch_pdl(colsum_kernel, dim3(blocks_for(d, 32)), dim3(32, 16), 0, st, (const float*)partial, parts, d, dg);
 }
 
 cudaError_t launch_geglu_fwd(int dtype, int act, const void* h, void* hg, int rows, int F, cudaStream_t st) {

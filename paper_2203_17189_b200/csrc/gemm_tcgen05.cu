@@ -578,10 +578,15 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   cluster_sync_all();                 // barriers of both CTAs exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
+  // Programmatic dependent launch: the next kernel of the stream (if it was launched that way) may bring its CTAs
+  // in and run its own set-up while this grid drains; the threads of this kernel that touch global memory wait here
+  // for the grid before it (no-ops under an ordinary launch).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
     if (lane == 0) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
@@ -656,6 +661,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const int g0 = ch < 2 ? ch * 2 : 4, g1 = ch < 2 ? ch * 2 + 2 : 4;
     int it = 0;
     bool ok = true;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     WorkIter wi(p, k_blocks, pair, n_pairs);
     Work w;
     for (; ok && wi.next(w); ++it) {
@@ -808,8 +814,13 @@ cudaError_t launch2(const GemmArgs& g, const CUtensorMap& ma, const CUtensorMap&
   } else if (tiles < pairs) {
     pairs = tiles;
   }
-  kern<<<2 * pairs, kThreads2, Smem2::kTotal, st>>>(ma, mb, p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(kThreads2); cfg.dynamicSmemBytes = Smem2::kTotal; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, ma, mb, p);
 }
 
 // 256 x 256 tiles on CTA pairs: boxes are 128 rows (K-major) or 64 x 64 (MN-major), as for BN = 128
