@@ -74,7 +74,7 @@ def attention_flops(c, B=None):
 # source the capture ran: keyed by the SHA-1 of csrc/gemm_tcgen05.cu, anything else reports null.
 GEMM_DRAM_TRAFFIC = {
     # "sha1 of gemm_tcgen05.cu": {"xl": bytes per launch averaged over the 795 GEMM launches of a step}
-    "46d6c3b22abd5a4767b897f4827e6b010dffc90c": {"xl": 290.3e6},
+    "45b35e45ff2aa93c561dcf57cd08107b73f57855": {"xl": 290.1e6},
 }
 
 
